@@ -1,0 +1,231 @@
+"""Seeded synthetic inputs for paged-KV decode attention.
+
+Shared by the tests, the benchmark and the smoke check; holds none of the
+method's arithmetic (no dot products, no softmax) -- only random tensors, context
+lengths and block tables shaped like the decoding of long reasoning traces by a
+32B-class GQA model (64 query heads, 8 KV heads, head_dim 128, bf16; traces of a
+few thousand to 32,768 tokens, several samples per prompt).
+
+Conventions
+-----------
+* pools are ``[num_pages][Hkv][P][D]`` bf16; K and V share page ids;
+* the pool holds exactly ``sum_b ceil(len_b / P)`` pages; the i-th logical page
+  in sequence-major order lives in physical page ``perm[i]`` (identity when the
+  table is "contiguous", one seeded permutation otherwise);
+* unused block-table entries are -1; slots at or beyond a sequence's length in its
+  last page are filled with bf16 NaN in K and V (a correct kernel never lets them
+  reach its output);
+* "uniform in [a, b]" is integer, both ends inclusive; "log-uniform" is
+  ``round(a * (b/a)**u)``, u ~ U[0,1), clamped to [a, b];
+* every random draw comes from a counter-based generator (numpy Philox for
+  lengths and permutations, torch's Philox-backed generator for tensors) seeded
+  from the workload's seed and a per-tensor stream id, so a workload is a pure
+  function of (name, seed, device type).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+NUM_Q_HEADS = 64
+NUM_KV_HEADS = 8
+HEAD_DIM = 128
+
+
+@dataclass
+class Spec:
+    name: str
+    batch: int
+    page_size: int
+    lengths: tuple            # ("const", n) | ("uniform", a, b) | ("loguniform", a, b) | ("skew", long, a, b) | ("list", [...])
+    permute_pages: bool = True
+    q_std: float = 1.0
+    k_outlier_prob: float = 0.0   # probability that a token position's K rows (all KV heads) are scaled
+    k_outlier_scale: float = 20.0
+    seed: int = 0
+    num_q_heads: int = NUM_Q_HEADS
+    num_kv_heads: int = NUM_KV_HEADS
+    head_dim: int = HEAD_DIM
+
+
+# The five decode configurations (batch / context mix / page size), seeds 73561..73565.
+SPECS = {
+    "cfg1_b1_ctx512_p16": Spec("cfg1_b1_ctx512_p16", 1, 16, ("const", 512), permute_pages=False, seed=73561),
+    "cfg2_b16_u1k_8k_p16": Spec("cfg2_b16_u1k_8k_p16", 16, 16, ("uniform", 1024, 8192), seed=73562),
+    "cfg3_b64_ctx16384_p64": Spec("cfg3_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563),
+    "cfg4_b256_logu2k_32k_p64": Spec("cfg4_b256_logu2k_32k_p64", 256, 64, ("loguniform", 2048, 32768), seed=73564),
+    "cfg5_b32_skew128k_p64": Spec("cfg5_b32_skew128k_p64", 32, 64, ("skew", 131072, 256, 4096),
+                                  k_outlier_prob=0.01, seed=73565),
+}
+
+
+@dataclass
+class Workload:
+    spec: Spec
+    q: torch.Tensor            # [B][Hq][D] bf16
+    k_pages: torch.Tensor      # [pages][Hkv][P][D] bf16
+    v_pages: torch.Tensor
+    block_table: torch.Tensor  # [B][stride] int32
+    seq_lens: torch.Tensor     # [B] int32
+    scale: float
+    lens_host: np.ndarray = field(default=None)
+    table_host: np.ndarray = field(default=None)
+
+    @property
+    def num_pages(self) -> int:
+        return self.k_pages.shape[0]
+
+    @property
+    def kv_tokens(self) -> int:
+        return int(self.lens_host.sum())
+
+    def algorithmic_bytes(self) -> int:
+        """K+V bytes of every cached token, q/out/lse of every sequence, and the block-table
+        entries and lengths the operation must read."""
+        s = self.spec
+        per_token = 2 * s.num_kv_heads * s.head_dim * 2
+        per_seq = 2 * s.num_q_heads * s.head_dim * 2 + s.num_q_heads * 4
+        pages = int(np.sum((self.lens_host + s.page_size - 1) // s.page_size))
+        return self.kv_tokens * per_token + s.batch * (per_seq + 4) + pages * 4
+
+
+def _rng(seed: int, stream: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[seed, stream]))
+
+
+def make_lengths(spec: Spec) -> np.ndarray:
+    r = _rng(spec.seed, 1)
+    kind = spec.lengths[0]
+    B = spec.batch
+    if kind == "const":
+        lens = np.full(B, spec.lengths[1], dtype=np.int64)
+    elif kind == "list":
+        lens = np.asarray(spec.lengths[1], dtype=np.int64)
+        assert lens.shape == (B,)
+    elif kind == "uniform":
+        _, a, b = spec.lengths
+        lens = r.integers(a, b + 1, size=B)
+    elif kind == "loguniform":
+        _, a, b = spec.lengths
+        u = r.random(B)
+        lens = np.clip(np.rint(a * (b / a) ** u), a, b).astype(np.int64)
+    elif kind == "skew":
+        _, long_len, a, b = spec.lengths
+        lens = r.integers(a, b + 1, size=B)
+        lens[0] = long_len
+    else:
+        raise ValueError(kind)
+    return lens.astype(np.int32)
+
+
+def make_block_table(spec: Spec, lens: np.ndarray, stride: int | None = None):
+    """Returns (table [B][stride] int32 with -1 tails, num_pages)."""
+    P = spec.page_size
+    pages_per_seq = (lens.astype(np.int64) + P - 1) // P
+    total = int(pages_per_seq.sum())
+    perm = np.arange(total, dtype=np.int64)
+    if spec.permute_pages:
+        perm = _rng(spec.seed, 2).permutation(total)
+    width = max(1, int(pages_per_seq.max())) if stride is None else stride
+    table = np.full((len(lens), width), -1, dtype=np.int32)
+    at = 0
+    for b, n in enumerate(pages_per_seq):
+        table[b, :n] = perm[at:at + n]
+        at += n
+    return table, max(total, 1)
+
+
+def _normal_bf16(shape, std, gen, device, chunk_elems=1 << 28):
+    """bf16 tensor of N(0, std^2) values rounded to nearest-even, drawn chunk by chunk."""
+    out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    flat = out.view(-1)
+    n = flat.numel()
+    for at in range(0, n, chunk_elems):
+        m = min(chunk_elems, n - at)
+        x = torch.randn(m, generator=gen, device=device, dtype=torch.float32)
+        if std != 1.0:
+            x *= std
+        flat[at:at + m] = x.to(torch.bfloat16)
+    return out
+
+
+def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = None) -> Workload:
+    if isinstance(spec, str):
+        spec = SPECS[spec]
+    device = torch.device(device)
+    lens = make_lengths(spec)
+    table, num_pages = make_block_table(spec, lens, table_stride)
+    Hq, Hkv, D, P = spec.num_q_heads, spec.num_kv_heads, spec.head_dim, spec.page_size
+
+    def gen(stream):
+        g = torch.Generator(device=device)
+        g.manual_seed(spec.seed * 1000 + stream)
+        return g
+
+    q = _normal_bf16((spec.batch, Hq, D), spec.q_std, gen(3), device)
+    v = _normal_bf16((num_pages, Hkv, P, D), 1.0, gen(5), device)
+    if spec.k_outlier_prob > 0.0:
+        # outliers are per token position: the K rows of all KV heads of that slot are
+        # scaled in fp32 before the rounding to bf16
+        k = torch.empty((num_pages, Hkv, P, D), dtype=torch.bfloat16, device=device)
+        gk, gm = gen(4), gen(6)
+        step = max(1, (1 << 26) // (Hkv * P * D))
+        for at in range(0, num_pages, step):
+            m = min(step, num_pages - at)
+            x = torch.randn((m, Hkv, P, D), generator=gk, device=device, dtype=torch.float32)
+            hit = torch.rand((m, 1, P, 1), generator=gm, device=device) < spec.k_outlier_prob
+            x = torch.where(hit, x * spec.k_outlier_scale, x)
+            k[at:at + m] = x.to(torch.bfloat16)
+    else:
+        k = _normal_bf16((num_pages, Hkv, P, D), 1.0, gen(4), device)
+
+    # poison the slots past each sequence's end in its last page
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16, device=device)
+    for b, n in enumerate(lens):
+        n = int(n)
+        if n % P:
+            page = int(table[b, (n - 1) // P])
+            k[page, :, n % P:, :] = nan
+            v[page, :, n % P:, :] = nan
+
+    return Workload(
+        spec=spec, q=q, k_pages=k, v_pages=v,
+        block_table=torch.from_numpy(table).to(device),
+        seq_lens=torch.from_numpy(lens).to(device),
+        scale=float(np.float32(1.0) / np.sqrt(np.float32(D))),
+        lens_host=lens, table_host=table)
+
+
+def tiny_spec(name, lens, page_size, seed, permute=True, **kw) -> Spec:
+    """A small hand-sized workload with the given context lengths."""
+    return Spec(name, len(lens), page_size, ("list", list(lens)), permute_pages=permute, seed=seed, **kw)
+
+
+def gather_sequences(w: Workload, seqs) -> Workload:
+    """A host-side copy of the given sequences only: their pages are renumbered
+    0..n-1 in logical order.  Lets a CPU checker look at a few sequences of a
+    workload whose pools are too large to copy whole."""
+    seqs = list(seqs)
+    P = w.spec.page_size
+    lens = w.lens_host[seqs]
+    pages_per_seq = (lens.astype(np.int64) + P - 1) // P
+    phys = np.concatenate([w.table_host[b, :n] for b, n in zip(seqs, pages_per_seq)]).astype(np.int64) \
+        if len(seqs) else np.zeros(0, np.int64)
+    idx = torch.from_numpy(phys).to(w.k_pages.device)
+    k = w.k_pages.index_select(0, idx).cpu()
+    v = w.v_pages.index_select(0, idx).cpu()
+    width = max(1, int(pages_per_seq.max())) if len(seqs) else 1
+    table = np.full((len(seqs), width), -1, dtype=np.int32)
+    at = 0
+    for i, n in enumerate(pages_per_seq):
+        table[i, :n] = np.arange(at, at + n)
+        at += n
+    sub = Spec(w.spec.name + "_subset", len(seqs), P, ("list", [int(x) for x in lens]),
+               seed=w.spec.seed, num_q_heads=w.spec.num_q_heads, num_kv_heads=w.spec.num_kv_heads,
+               head_dim=w.spec.head_dim)
+    return Workload(spec=sub, q=w.q[seqs].cpu(), k_pages=k, v_pages=v,
+                    block_table=torch.from_numpy(table), seq_lens=torch.from_numpy(lens.astype(np.int32)),
+                    scale=w.scale, lens_host=lens.astype(np.int32), table_host=table)
