@@ -1,0 +1,386 @@
+"""Benchmark of one decode-attention step (plan + split-KV partial + LSE combine) through the
+C ABI on seeded synthetic long-trace workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One JSON line on stdout (rank 0).  `value` is the algorithmic bytes of the step (K and V of
+every cached token, q/out/lse, used table entries) divided by the device time of the whole
+step with all inputs resident in HBM; `e2e` is the same through the host-buffer entry point
+with every host<->device copy inside the timed region; `roofline` times the partial kernel
+alone with events the library records around it; `cpu_baseline` is the fp64 CPU oracle on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attention_kv_bandwidth"
+UNIT = "GB/s"
+DEFAULT_WORKLOAD = "cfg3_b64_ctx16384_p64"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--kernel", type=int, default=0, help="0 tensor-core partial kernel, 1 scalar-FMA")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--ranges-per-cta", type=int, default=0)
+    ap.add_argument("--min-range-tiles", type=int, default=0)
+    ap.add_argument("--num-ranges", type=int, default=0)
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def mark(self):
+        return time.time()
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if (t0 is None or t >= t0 - 0.05) and (t1 is None or t <= t1 + 0.1)]
+        if not rows:
+            rows = [l for _, l in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            parts = [x.strip() for x in r.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample_throughput(w_host, seqs, threads):
+    """Times the CPU oracle (as it stands) on whole sequences handed to a thread pool."""
+    from concurrent.futures import ThreadPoolExecutor
+    import oracle
+    qb = oracle._u16(w_host.q); kb = oracle._u16(w_host.k_pages); vb = oracle._u16(w_host.v_pages)
+    tb = oracle._i32(w_host.block_table); lb = oracle._i32(w_host.seq_lens)
+    Hq = w_host.spec.num_q_heads
+    units = [(b, h0) for b in seqs for h0 in range(0, Hq, 8)]      # one KV-head group per unit
+
+    def one(u):
+        b, h0 = u
+        oracle.decode_attn(qb, kb, vb, tb, lb, w_host.scale, seqs=(b, b + 1), heads=(h0, h0 + 8))
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(one, units))
+    return time.perf_counter() - t0
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(w, target_seconds):
+    """Oracle throughput on a bounded sample of the workload's sequences (all 64 heads each)."""
+    import numpy as np
+    import synth
+    cores = host_cores()
+    order = np.random.default_rng(7).permutation(w.spec.batch).tolist()
+    # calibrate on one KV-head group of the first sampled sequence
+    first = synth.gather_sequences(w, order[:1])
+    import oracle
+    oracle.build()
+    t0 = time.perf_counter()
+    oracle.decode_attn(first.q, first.k_pages, first.v_pages, first.block_table, first.seq_lens,
+                       first.scale, seqs=(0, 1), heads=(0, 8))
+    cal = time.perf_counter() - t0
+    per_token_core = cal * 8 / max(1, int(first.lens_host[0]))        # seconds per KV token on one core
+    budget_tokens = target_seconds * cores / max(per_token_core, 1e-12)
+    seqs, tok = [], 0
+    for b in order:
+        seqs.append(b)
+        tok += int(w.lens_host[b])
+        if tok >= budget_tokens:
+            break
+    sub = synth.gather_sequences(w, seqs)
+    dt = oracle_sample_throughput(sub, list(range(len(seqs))), cores)
+    nbytes = sub.algorithmic_bytes()
+    return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(seqs)} of {w.spec.batch} sequences ({tok} of {w.kv_tokens} KV tokens), all 64 heads, "
+                      f"{dt:.1f} s wall", "kv_tokens_per_s": tok / dt}
+
+
+def run_reference(args):
+    """The oracle timed on the host cores; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    import synth
+    # the sample is built from the workload's lengths without building its full pools
+    spec = synth.SPECS[args.workload]
+    lens = synth.make_lengths(spec)
+    cores = host_cores()
+    # bounded sample: sequences in a seeded order, sized by a one-group calibration
+    order = np.random.default_rng(7).permutation(spec.batch).tolist()
+    probe = synth.make_workload(synth.tiny_spec("probe", (int(lens[order[0]]),), spec.page_size, spec.seed,
+                                                q_std=spec.q_std), "cpu")
+    import oracle
+    oracle.build()
+    t0 = time.perf_counter()
+    oracle.decode_attn(probe.q, probe.k_pages, probe.v_pages, probe.block_table, probe.seq_lens, probe.scale,
+                       seqs=(0, 1), heads=(0, 8))
+    per_token_core = (time.perf_counter() - t0) * 8 / max(1, int(lens[order[0]]))
+    total_steps = args.steps + args.warmup
+    budget_tokens = (120.0 / total_steps) * cores / max(per_token_core, 1e-12)
+    seqs, tok = [], 0
+    for b in order:
+        seqs.append(b); tok += int(lens[b])
+        if tok >= budget_tokens:
+            break
+    sample = synth.make_workload(
+        synth.tiny_spec("sample", [int(lens[b]) for b in seqs], spec.page_size, spec.seed, q_std=spec.q_std,
+                        k_outlier_prob=spec.k_outlier_prob), "cpu")
+    for _ in range(args.warmup):
+        oracle_sample_throughput(sample, list(range(len(seqs))), cores)
+    t = [oracle_sample_throughput(sample, list(range(len(seqs))), cores) for _ in range(args.steps)]
+    dt = sum(t) / len(t)
+    nbytes = sample.algorithmic_bytes()
+    value = nbytes / dt / 1e9
+    desc = (f"{len(seqs)} of {spec.batch} sequences ({tok} of {int(lens.sum())} KV tokens), all 64 heads, per step")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "kv_tokens_per_s": tok / dt, "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import synth
+    import paper_2510_07356_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    # every rank decodes its own batch of the same shape (replicas, no data-path collective)
+    spec = synth.SPECS[args.workload]
+    if world > 1:
+        from dataclasses import replace
+        spec = replace(spec, seed=spec.seed + 100 * rank)
+    w = synth.make_workload(spec, dev)
+    attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
+    attn.set_option(P.CONCUR_OPT_KERNEL, args.kernel)
+    attn.set_option(P.CONCUR_OPT_RANGES_PER_CTA, args.ranges_per_cta)
+    attn.set_option(P.CONCUR_OPT_MIN_RANGE_TILES, args.min_range_tiles)
+    attn.set_option(P.CONCUR_OPT_NUM_RANGES, args.num_ranges)
+    out = torch.empty_like(w.q)
+    lse = torch.empty((spec.batch, spec.num_q_heads), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    nbytes = w.algorithmic_bytes()
+    kv_bytes = w.kv_tokens * 2 * spec.num_kv_heads * spec.head_dim * 2
+    flush_needed = kv_bytes < 512 * 1024 * 1024          # inputs not well above the 126 MB L2
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if flush_needed else None
+
+    def step():
+        attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale, out=out, lse=lse)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(max(3, args.warmup)):
+        if flush_buf is not None:
+            flush_buf.zero_()
+        step()
+    barrier()
+    assert attn.status() == 0, "device-side flags set during warm-up"
+
+    # ---- timed region: K whole steps; events around each step and around its partial kernel
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    for row in ev:                       # materialise the cudaEvent_t handles
+        for e in row:
+            e.record(stream)
+    torch.cuda.synchronize(dev)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    barrier()
+    t_mark0 = time.time()
+    for i in range(K):
+        if flush_buf is not None:
+            flush_buf.zero_()
+        attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, ev[i][1].cuda_event)
+        attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, ev[i][2].cuda_event)
+        ev[i][0].record(stream)
+        step()
+        ev[i][3].record(stream)
+    barrier()
+    t_mark1 = time.time()
+    clocks = sampler.stop(t_mark0, t_mark1) if rank == 0 else None
+    attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, 0)
+    attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, 0)
+    step_ms = [ev[i][0].elapsed_time(ev[i][3]) for i in range(K)]
+    part_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)]
+    ms_per_step = sum(step_ms) / K
+    part_ms_avg = sum(part_ms) / K
+    if world > 1:
+        t = torch.tensor([ms_per_step, part_ms_avg], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, part_ms_avg = t.tolist()
+    flags = attn.status()
+    R, W, _ = attn.last_plan()
+
+    # ---- end to end: host buffers, every copy inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        hq, hk, hv, hbt, hsl = pin(w.q), pin(w.k_pages), pin(w.v_pages), pin(w.block_table), pin(w.seq_lens)
+        hout = torch.empty(w.q.shape, dtype=torch.bfloat16).pin_memory()
+        hlse = torch.empty((spec.batch, spec.num_q_heads), dtype=torch.float32).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hbt, hsl))
+        d2h = hout.numel() * 2 + hlse.numel() * 4
+
+        def host_step():
+            P.concur_decode_attn_host(attn.handle, hq, hk, hv, hbt, hsl, w.scale, hout, hlse, spec.batch,
+                                      hk.shape[0], hbt.shape[1], stream.cuda_stream)
+        host_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            host_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = t.item()
+        e2e = {"value": world * nbytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+               "entry": "concur_decode_attn_host"}
+        assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), "host path differs from device path"
+        del hq, hk, hv
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
+    achieved = nbytes / (part_ms_avg * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
+                   "heads": "64q/8kv", "head_dim": 128, "algorithmic_bytes": nbytes,
+                   "l2": "flushed between steps" if flush_needed else "inputs larger than L2",
+                   "kernel": "mma" if args.kernel == 0 else "scalar", "ranges": R, "tiles": W,
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+        "kv_tokens_per_s": world * w.kv_tokens / (ms_per_step * 1e-3),
+        "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
+        "frac_of_measured_copy": value / world / peak,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "partial", "ms": part_ms_avg,
+                     "ms_min": min(part_ms)},
+        "step_ms_min": min(step_ms),
+        "e2e": e2e, "gpu_launches": 3 * K, "clocks": clocks, "device_flags": flags,
+    }
+    if not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

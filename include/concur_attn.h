@@ -1,0 +1,177 @@
+/*
+ * concur_attn -- paged-KV grouped-query decode attention for NVIDIA B200 (sm_100a).
+ *
+ * One call computes one decode step of one layer:  for every sequence b of the batch
+ * and every query head h (KV head g = h / (Hq/Hkv)), over the n = seq_lens[b] tokens
+ * cached for that sequence,
+ *
+ *     s_j   = scale * <q[b][h], K[token j of b][g]>
+ *     out   = sum_j softmax(s)_j * V[token j of b][g]          (bf16, round-to-nearest-even)
+ *     lse   = ln sum_j exp(s_j)                                  (fp32, natural log)
+ *     n = 0:  out = 0, lse = -inf.
+ *
+ * This is the attention step of the batched autoregressive decoding of long reasoning
+ * traces on which the ConCuR pipeline (arXiv 2510.07356) spends its generation time:
+ * five samples for each of 18,162 tasks by a 32B GQA model (Sec. 3.3), ten per task in
+ * evaluation (Sec. 4.1), traces of 4,000-8,500 tokens and more (Tables 3 and 4) under a
+ * 32,768-token limit (Sec. 4.1).  The paper states no formula for it; the definition
+ * above is the standard one.
+ *
+ * Method: a plan kernel cuts the batch's KV tiles into ranges of near-equal size
+ * (split-KV), a partial kernel streams each K/V tile from HBM once for all query heads
+ * of its GQA group with an fp32 online softmax, and a combine kernel merges the partial
+ * results of sequences that were split, by their log-sum-exp.
+ *
+ * Memory layout (all device memory unless a parameter says otherwise; caller-owned):
+ *     q            bf16  [batch][Hq][D]
+ *     k_pages      bf16  [num_pages][Hkv][P][D]        one (page, head) tile is contiguous
+ *     v_pages      bf16  same shape; K and V of a token share page id and slot
+ *     block_table  int32 [batch][block_table_stride]   logical page i of b -> physical page
+ *     seq_lens     int32 [batch]
+ *     out          bf16  [batch][Hq][D]
+ *     lse          fp32  [batch][Hq]
+ * Token j of sequence b is slot j % P of page block_table[b][j / P].  Table entries at
+ * or beyond ceil(n/P), and slots at or beyond n in the last page, are never read into a
+ * result (they may hold anything, NaN included).
+ *
+ * Conventions: every function returns CONCUR_OK (0) or a negative concur_status_t; none
+ * throws, aborts or prints.  No pointer is retained after a call returns.  The library
+ * has no CPU fallback: without a CUDA device every call fails with CONCUR_ERR_CUDA.
+ */
+#ifndef CONCUR_ATTN_H_
+#define CONCUR_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CONCUR_OK = 0,
+    CONCUR_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, negative size, unknown option   */
+    CONCUR_ERR_UNSUPPORTED = -2,   /* geometry outside what the kernels are built for             */
+    CONCUR_ERR_TOO_LARGE = -3,     /* batch, table stride or workspace beyond the handle's limits */
+    CONCUR_ERR_CUDA = -4,          /* a CUDA runtime or driver call failed (no device, launch)    */
+    CONCUR_ERR_OOM = -5            /* device allocation failed                                     */
+} concur_status_t;
+
+/* Sticky device-side condition bits reported by concur_attn_status. */
+#define CONCUR_FLAG_BAD_PAGE_ID 1u  /* a used block-table entry was outside [0, num_pages): clamped    */
+#define CONCUR_FLAG_BAD_SEQ_LEN 2u  /* a seq_lens entry was outside [0, stride*P]: clamped             */
+#define CONCUR_FLAG_WAIT_LIMIT  4u  /* an in-kernel wait gave up; results of that call are invalid      */
+
+/* Option keys for concur_attn_set_option (tuning and tests; defaults are chosen per call). */
+#define CONCUR_OPT_KERNEL      1    /* 0 = tensor-core partial kernel (default), 1 = scalar-FMA kernel */
+#define CONCUR_OPT_NUM_RANGES  2    /* force the number of split-KV ranges; 0 = heuristic              */
+#define CONCUR_OPT_GRID_CTAS   3    /* force the partial kernel's grid size; 0 = one wave of the GPU    */
+#define CONCUR_OPT_RANGES_PER_CTA 4 /* heuristic's target ranges per CTA; 0 = built-in default          */
+#define CONCUR_OPT_MIN_RANGE_TILES 5/* heuristic's smallest range, in 64-token tiles; 0 = default       */
+#define CONCUR_OPT_EVENT_BEFORE_PARTIAL 6 /* a cudaEvent_t (as an integer) recorded on the call's stream
+                                             just before the partial kernel; 0 = none.  For timing
+                                             that kernel alone; the event stays the caller's.          */
+#define CONCUR_OPT_EVENT_AFTER_PARTIAL  7 /* likewise, just after the partial kernel                    */
+
+typedef struct concur_attn concur_attn_t;   /* opaque; owns its workspace and nothing else */
+
+typedef struct {
+    int32_t num_q_heads;        /* Hq; supported: 64                                            */
+    int32_t num_kv_heads;       /* Hkv; supported: 8 (group size Hq/Hkv = 8)                    */
+    int32_t head_dim;           /* D; supported: 128                                            */
+    int32_t page_size;          /* P; supported: 16, 32, 64 tokens                              */
+    int32_t max_batch;          /* largest `batch` any call will pass (1 .. 65536)              */
+    int32_t max_pages_per_seq;  /* largest `block_table_stride` any call will pass             */
+    int32_t device;             /* CUDA device ordinal                                          */
+    int32_t reserved;           /* must be 0                                                    */
+    void*   workspace;          /* optional device memory (256-byte aligned) of at least
+                                   concur_attn_workspace_bytes(); NULL: the library allocates  */
+    size_t  workspace_bytes;    /* size of `workspace`; ignored when it is NULL                */
+} concur_attn_config_t;
+
+/*
+ * Bytes of device workspace a handle with this configuration needs (split-KV partial
+ * results, the plan's tables, counters).  Host function, no CUDA call.  Returns 0 for an
+ * invalid or unsupported configuration.
+ */
+size_t concur_attn_workspace_bytes(const concur_attn_config_t* cfg);
+
+/*
+ * Creates a handle on cfg->device.  Checks the geometry (CONCUR_ERR_UNSUPPORTED), the
+ * limits (CONCUR_ERR_INVALID_ARG), takes or allocates the workspace (CONCUR_ERR_OOM,
+ * CONCUR_ERR_TOO_LARGE if a caller-supplied one is too small) and clears it on the
+ * device's default stream (synchronously).  *handle is written only on success.
+ */
+int concur_attn_create(const concur_attn_config_t* cfg, concur_attn_t** handle);
+
+/*
+ * One decode-attention step, enqueued on `cuda_stream` (a cudaStream_t; NULL = default
+ * stream).  Asynchronous: returns after the launches are queued, never synchronises, and
+ * reads seq_lens / block_table on the device only.  Calls on one handle must be
+ * stream-ordered with each other (they share the workspace).
+ *
+ *   q, k_pages, v_pages, out   device, 16-byte aligned, layouts as in the file header
+ *   block_table, seq_lens      device, 4-byte aligned
+ *   scale                      multiplies q.k before the softmax (1/sqrt(D) usually)
+ *   batch                      0 <= batch <= max_batch   (0: nothing is launched)
+ *   num_pages                  pages in each pool, >= 1
+ *   block_table_stride         int32 elements per table row, 1 .. max_pages_per_seq
+ *
+ * Errors: CONCUR_ERR_INVALID_ARG (null or misaligned pointer, bad size),
+ * CONCUR_ERR_TOO_LARGE (batch or stride above the handle's limits), CONCUR_ERR_CUDA
+ * (launch failure).  Bad *contents* never fault: a page id outside [0, num_pages) or a
+ * length outside [0, stride*P] is clamped and recorded (see concur_attn_status); the
+ * affected sequences' results are then unspecified but finite memory is all that is read.
+ */
+int concur_decode_attn(concur_attn_t* handle,
+                       const void* q, const void* k_pages, const void* v_pages,
+                       const int32_t* block_table, const int32_t* seq_lens,
+                       float scale, void* out, float* lse,
+                       int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                       void* cuda_stream);
+
+/*
+ * The same step for callers whose tensors live in HOST memory (pinned memory gives
+ * asynchronous copies).  Every pointer is a host pointer with the layouts above; the
+ * library copies the inputs into device staging buffers that it owns (allocated on first
+ * use and grown when a call needs more: cudaMalloc inside this call), runs the three
+ * kernels, copies out / lse back and synchronises the stream before returning.
+ * Errors as for concur_decode_attn, plus CONCUR_ERR_OOM.
+ */
+int concur_decode_attn_host(concur_attn_t* handle,
+                            const void* q, const void* k_pages, const void* v_pages,
+                            const int32_t* block_table, const int32_t* seq_lens,
+                            float scale, void* out, float* lse,
+                            int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                            void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and returns, in *flags (host pointer), the OR of the
+ * CONCUR_FLAG_* conditions seen by any call on this handle since the last status call;
+ * the device word is then cleared.
+ */
+int concur_attn_status(concur_attn_t* handle, void* cuda_stream, uint32_t* flags);
+
+/* Sets a CONCUR_OPT_* value for later calls on this handle.  Unknown key or a value out
+ * of range: CONCUR_ERR_INVALID_ARG. */
+int concur_attn_set_option(concur_attn_t* handle, int32_t key, int64_t value);
+
+/*
+ * For tests and load-balance reports: copies the plan of the most recent call to the
+ * host (synchronises `cuda_stream`).  *num_ranges and *total_tiles receive the split-KV
+ * range count and the number of (KV head, 64-token tile) units; range_start (host,
+ * capacity `cap` int32s, may be NULL) receives min(cap, num_ranges+1) range boundaries.
+ */
+int concur_attn_last_plan(concur_attn_t* handle, void* cuda_stream, int32_t* num_ranges,
+                          int32_t* total_tiles, int32_t* range_start, int32_t cap);
+
+/* Frees the handle and any memory the library allocated for it.  NULL is accepted. */
+int concur_attn_destroy(concur_attn_t* handle);
+
+/* Static, never-NULL description of a status code. */
+const char* concur_attn_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONCUR_ATTN_H_ */

@@ -1,0 +1,176 @@
+"""ctypes binding of libconcur_attn.so: the same names as include/concur_attn.h.
+
+Argument marshalling only -- every step of the decode-attention path (plan, partial,
+combine) runs in the library's CUDA kernels.  There is no fallback: if the shared
+library is missing or was not built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_LIB_PATH = Path(__file__).resolve().parent / "libconcur_attn.so"
+
+CONCUR_OK = 0
+CONCUR_ERR_INVALID_ARG = -1
+CONCUR_ERR_UNSUPPORTED = -2
+CONCUR_ERR_TOO_LARGE = -3
+CONCUR_ERR_CUDA = -4
+CONCUR_ERR_OOM = -5
+
+CONCUR_FLAG_BAD_PAGE_ID = 1
+CONCUR_FLAG_BAD_SEQ_LEN = 2
+CONCUR_FLAG_WAIT_LIMIT = 4
+
+CONCUR_OPT_KERNEL = 1
+CONCUR_OPT_NUM_RANGES = 2
+CONCUR_OPT_GRID_CTAS = 3
+CONCUR_OPT_RANGES_PER_CTA = 4
+CONCUR_OPT_MIN_RANGE_TILES = 5
+CONCUR_OPT_EVENT_BEFORE_PARTIAL = 6
+CONCUR_OPT_EVENT_AFTER_PARTIAL = 7
+
+EXPORTS = (
+    "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",
+    "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
+    "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
+)
+
+
+class concur_attn_config_t(ctypes.Structure):
+    _fields_ = [
+        ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+        ("max_batch", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
+        ("device", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+def _load() -> ctypes.CDLL:
+    if not _LIB_PATH.exists():
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2510_07356_b200.build` "
+            "(nvcc, sm_100a). There is no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i32, i32p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)
+    cfgp = ctypes.POINTER(concur_attn_config_t)
+    lib.concur_attn_workspace_bytes.restype = ctypes.c_size_t
+    lib.concur_attn_workspace_bytes.argtypes = [cfgp]
+    lib.concur_attn_create.restype = ctypes.c_int
+    lib.concur_attn_create.argtypes = [cfgp, ctypes.POINTER(vp)]
+    decode_args = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, vp]
+    lib.concur_decode_attn.restype = ctypes.c_int
+    lib.concur_decode_attn.argtypes = decode_args
+    lib.concur_decode_attn_host.restype = ctypes.c_int
+    lib.concur_decode_attn_host.argtypes = decode_args
+    lib.concur_attn_status.restype = ctypes.c_int
+    lib.concur_attn_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.concur_attn_set_option.restype = ctypes.c_int
+    lib.concur_attn_set_option.argtypes = [vp, i32, ctypes.c_int64]
+    lib.concur_attn_last_plan.restype = ctypes.c_int
+    lib.concur_attn_last_plan.argtypes = [vp, vp, i32p, i32p, i32p, i32]
+    lib.concur_attn_destroy.restype = ctypes.c_int
+    lib.concur_attn_destroy.argtypes = [vp]
+    lib.concur_attn_strerror.restype = ctypes.c_char_p
+    lib.concur_attn_strerror.argtypes = [ctypes.c_int]
+    return lib
+
+
+lib = _load()
+
+
+class ConcurError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {concur_attn_strerror(code)} ({code})")
+
+
+def concur_attn_strerror(code: int) -> str:
+    return lib.concur_attn_strerror(int(code)).decode()
+
+
+def make_config(page_size: int, max_batch: int, max_pages_per_seq: int, device: int = 0,
+                num_q_heads: int = 64, num_kv_heads: int = 8, head_dim: int = 128,
+                workspace: int = 0, workspace_bytes: int = 0) -> concur_attn_config_t:
+    return concur_attn_config_t(num_q_heads, num_kv_heads, head_dim, page_size, max_batch,
+                                max_pages_per_seq, device, 0, workspace or None, workspace_bytes)
+
+
+def concur_attn_workspace_bytes(cfg: concur_attn_config_t) -> int:
+    return int(lib.concur_attn_workspace_bytes(ctypes.byref(cfg)))
+
+
+def concur_attn_create(cfg: concur_attn_config_t) -> int:
+    """Returns the handle as an integer address; raises ConcurError on failure."""
+    h = ctypes.c_void_p()
+    rc = lib.concur_attn_create(ctypes.byref(cfg), ctypes.byref(h))
+    if rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_attn_create")
+    return h.value
+
+
+def _addr(x) -> int:
+    """Device or host address of a torch tensor / numpy array / int."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    return x.ctypes.data
+
+
+def _decode(fn, name, handle, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
+            batch, num_pages, block_table_stride, stream, check):
+    rc = fn(handle, _addr(q), _addr(k_pages), _addr(v_pages), _addr(block_table), _addr(seq_lens),
+            ctypes.c_float(scale), _addr(out), _addr(lse), batch, num_pages, block_table_stride,
+            stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, name)
+    return rc
+
+
+def concur_decode_attn(handle, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
+                       batch, num_pages, block_table_stride, stream=0, check=True) -> int:
+    """Device tensors (or raw device addresses); `stream` is a cudaStream_t as an int."""
+    return _decode(lib.concur_decode_attn, "concur_decode_attn", handle, q, k_pages, v_pages,
+                   block_table, seq_lens, scale, out, lse, batch, num_pages, block_table_stride,
+                   stream, check)
+
+
+def concur_decode_attn_host(handle, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
+                            batch, num_pages, block_table_stride, stream=0, check=True) -> int:
+    """Host tensors (pinned for asynchronous copies); synchronises before returning."""
+    return _decode(lib.concur_decode_attn_host, "concur_decode_attn_host", handle, q, k_pages,
+                   v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
+                   block_table_stride, stream, check)
+
+
+def concur_attn_status(handle, stream=0) -> int:
+    flags = ctypes.c_uint32(0)
+    rc = lib.concur_attn_status(handle, stream or None, ctypes.byref(flags))
+    if rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_attn_status")
+    return flags.value
+
+
+def concur_attn_set_option(handle, key: int, value: int, check=True) -> int:
+    rc = lib.concur_attn_set_option(handle, key, value)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_attn_set_option")
+    return rc
+
+
+def concur_attn_last_plan(handle, stream=0, cap: int = 8192):
+    """Returns (num_ranges, total_tiles, range_start list) of the most recent call."""
+    n, w = ctypes.c_int32(0), ctypes.c_int32(0)
+    buf = (ctypes.c_int32 * cap)()
+    rc = lib.concur_attn_last_plan(handle, stream or None, ctypes.byref(n), ctypes.byref(w), buf, cap)
+    if rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_attn_last_plan")
+    return n.value, w.value, list(buf[: min(cap, n.value + 1)])
+
+
+def concur_attn_destroy(handle) -> int:
+    return lib.concur_attn_destroy(handle)

@@ -1,0 +1,114 @@
+// Shared declarations of the decode-attention kernels: the per-call parameter block,
+// the workspace layout and the range -> segment arithmetic of the split-KV plan.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace concur {
+
+constexpr int kHq = 64;          // query heads
+constexpr int kHkv = 8;          // KV heads
+constexpr int kGroup = 8;        // query heads per KV head
+constexpr int kD = 128;          // head dimension
+constexpr int kTile = 64;        // tokens per KV tile: the unit the plan counts in
+constexpr int kRowBytes = kD * 2;
+
+constexpr uint32_t kFlagBadPage = 1u;
+constexpr uint32_t kFlagBadLen = 2u;
+constexpr uint32_t kFlagWaitLimit = 4u;
+
+// Workspace header (int32 words).
+enum HeaderWord : int {
+    kHdrTotalTiles = 0,   // W: sum over (sequence, KV head) of ceil(len / 64)
+    kHdrNumRanges = 1,    // R: ranges the flat tile index space [0, W) is cut into
+    kHdrClaim = 2,        // next range to hand out (atomic)
+    kHdrStatus = 3,       // sticky CONCUR_FLAG_* bits
+    kHdrWords = 64
+};
+
+// Everything a launch needs.  Pointers are device pointers.
+struct DecodeParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_pages;
+    const __nv_bfloat16* v_pages;
+    const int32_t* block_table;
+    const int32_t* seq_lens;
+    __nv_bfloat16* out;
+    float* lse;
+    float scale_log2e;        // scale * log2(e): scores are kept in the base-2 domain
+    int32_t batch;
+    int32_t num_pages;
+    int32_t bt_stride;
+    int32_t page_size;
+    int32_t page_shift;       // log2(page_size)
+    // plan controls
+    int32_t grid_ctas;        // CTAs the partial kernel is launched with
+    int32_t forced_ranges;    // > 0: use exactly this many ranges (clamped to [1, min(W, max_ranges)])
+    int32_t ranges_per_cta;
+    int32_t min_range_tiles;
+    int32_t max_ranges;       // capacity of range_start / partial slots
+    // workspace
+    int32_t* hdr;             // [kHdrWords]
+    int32_t* tiles_prefix;    // [batch + 1] exclusive prefix of per-sequence tile counts
+    int32_t* range_start;     // [R + 1] boundaries in flat tile space
+    float* part_o;            // [2 * max_ranges][kGroup][kD] normalised partial outputs
+    float* part_lse;          // [2 * max_ranges][kGroup]     base-2 log-sum-exp of each partial
+};
+
+// The flat tile space lists, for sequence b = 0.., KV head g = 0..7, that unit's tiles:
+// unit (b, g) occupies [kHkv * prefix[b] + g * tiles_b, ... + tiles_b).
+struct Segment {
+    int32_t b, g;
+    int32_t tile0, tile1;     // tiles of the unit covered by this segment, [tile0, tile1)
+    int32_t tiles_b;          // tiles of the whole unit
+    int32_t slot;             // partial slot, or -1 when the segment covers the whole unit
+};
+
+// Largest b in [0, batch) with kHkv * prefix[b] <= x  (x < W).
+__device__ __forceinline__ int32_t find_sequence(const int32_t* __restrict__ prefix, int32_t batch, int32_t x) {
+    int32_t lo = 0, hi = batch;            // invariant: kHkv*prefix[lo] <= x < kHkv*prefix[hi]
+    while (hi - lo > 1) {
+        int32_t mid = (lo + hi) >> 1;
+        if (kHkv * prefix[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Largest r in [0, R) with range_start[r] <= x  (x < W).
+__device__ __forceinline__ int32_t find_range(const int32_t* __restrict__ range_start, int32_t R, int32_t x) {
+    int32_t lo = 0, hi = R;
+    while (hi - lo > 1) {
+        int32_t mid = (lo + hi) >> 1;
+        if (range_start[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Segment of range r that starts at flat tile x (range_start[r] <= x < range_start[r+1]).
+__device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix, int32_t batch,
+                                              int32_t r, int32_t x0, int32_t x1, int32_t x) {
+    Segment s;
+    s.b = find_sequence(prefix, batch, x);
+    int32_t base = kHkv * prefix[s.b];
+    s.tiles_b = prefix[s.b + 1] - prefix[s.b];
+    s.g = (x - base) / s.tiles_b;
+    int32_t unit_start = base + s.g * s.tiles_b;
+    int32_t unit_end = unit_start + s.tiles_b;
+    int32_t end = x1 < unit_end ? x1 : unit_end;
+    s.tile0 = x - unit_start;
+    s.tile1 = end - unit_start;
+    bool whole = (s.tile0 == 0) && (s.tile1 == s.tiles_b);
+    s.slot = whole ? -1 : 2 * r + (x > x0 ? 1 : 0);
+    return s;
+}
+
+// Host-side launchers (each enqueues on `stream` and returns the launch status).
+cudaError_t launch_plan(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_partial_scalar(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream);
+int partial_scalar_ctas_per_sm();
+
+}  // namespace concur

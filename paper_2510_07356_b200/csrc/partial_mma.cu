@@ -1,0 +1,551 @@
+// Split-KV partial kernel, tensor-core version (the default).
+//
+// One persistent CTA per SM: a producer warp streams K and V tiles (64 tokens x 128 dims,
+// 16 KB each) from the paged pools into a 6-stage shared-memory ring with TMA tensor
+// copies (128-byte swizzle, one copy per (page, KV head) chunk), four consumer warps
+// each own 16 tokens of every tile:
+//
+//   S^T[16 tok x 8 heads]  = K[16 tok x 128] . Q^T[128 x 8]        (8 mma.m16n8k16, bf16 -> fp32)
+//   online softmax in fp32, base-2 domain, per-warp running max / sum
+//   O^T[128 x 8 heads]    += V^T[128 x 16 tok] . P^T[16 tok x 8]   (8 mma.m16n8k16)
+//
+// so every K/V byte is fetched from HBM once and serves all 8 query heads of its GQA
+// group.  Tokens sit on the MMA's M dimension and the 8 heads fill its N = 8 exactly; the
+// probabilities go from accumulator layout to B-operand layout with two 8x8 register
+// transposes.  When a segment (a run of tiles of one (sequence, KV head) unit inside a
+// range of the plan) ends, the four warps' states are merged through shared memory and
+// written either straight to out/lse (the segment was the whole unit) or to a partial
+// slot for the combine kernel.
+//
+// The kernel is HBM-bound by design: ~32 issue slots per 8 KB of KV per warp; what matters
+// is the depth of the TMA ring (192 KB in flight per SM) and that nothing stalls the
+// producer (plan tables cached in shared memory, block-table entries prefetched 32 at a
+// time, the next range claimed while the current one streams).
+//
+// Every wait is bounded: a wait that exceeds its limit sets CONCUR_FLAG_WAIT_LIMIT, raises
+// a CTA-wide abort flag and every warp leaves; the producer first waits (bounded) for the
+// copies it has in flight.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace concur {
+
+namespace {
+
+constexpr int kStages = 6;
+constexpr int kConsumerWarps = 4;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kTileBytes = kTile * kRowBytes;             // 16 KB: one K or V tile
+constexpr int kQBytes = kGroup * kRowBytes;               // 2 KB: the 8 query rows of a group
+constexpr int kStageBytes = 2 * kTileBytes + kQBytes;     // K | V | Q
+constexpr int kMergeStride = kD + 4;                      // floats per head row in the merge buffer
+constexpr int kMergeBytes = kConsumerWarps * kGroup * kMergeStride * 4;
+constexpr int kSmemBatch = 511;                           // sequences whose plan rows are cached in smem
+constexpr uint64_t kWaitLimitNs = 2000000000ull;          // 2 s
+
+struct StageMeta {
+    int32_t b, g, slot;
+    int32_t n_valid;       // valid tokens in the tile (1..64); 0 = no more work
+    int32_t first, last;   // first / last tile of its segment
+    int32_t pad0, pad1;
+};
+
+struct Smem {
+    // offsets from the 1024-aligned base
+    static constexpr int kStagesOff = 0;
+    static constexpr int kMergeOff = kStages * kStageBytes;
+    static constexpr int kMlOff = kMergeOff + kMergeBytes;                       // [4 warps][8 heads][2]
+    static constexpr int kPrefixOff = kMlOff + kConsumerWarps * kGroup * 2 * 4;  // [kSmemBatch + 1]
+    static constexpr int kLenOff = kPrefixOff + (kSmemBatch + 1) * 4;            // [kSmemBatch + 1]
+    static constexpr int kMetaOff = kLenOff + (kSmemBatch + 1) * 4;
+    static constexpr int kBarOff = kMetaOff + kStages * (int)sizeof(StageMeta);  // full_k, full_v, empty, merge x2
+    static constexpr int kAbortOff = kBarOff + (3 * kStages + 2) * 8;
+    static constexpr int kTotal = kAbortOff + 16;
+};
+constexpr int kSmemBytes = Smem::kTotal + 1024;           // slack for the manual 1024-byte alignment
+static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false if the limit ran out or another warp raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    uint64_t t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int32_t row, uint32_t bar) {
+    // box {64 elements, P rows, 2 halves} at coordinates {0, row, 0}
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 1)
+partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    float* merge_o = reinterpret_cast<float*>(smem + Smem::kMergeOff);
+    float* merge_ml = reinterpret_cast<float*>(smem + Smem::kMlOff);
+    int32_t* sm_prefix = reinterpret_cast<int32_t*>(smem + Smem::kPrefixOff);
+    int32_t* sm_len = reinterpret_cast<int32_t*>(smem + Smem::kLenOff);
+    StageMeta* meta = reinterpret_cast<StageMeta*>(smem + Smem::kMetaOff);
+    volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(smem + Smem::kAbortOff);
+    const uint32_t bar_base = smem_base + Smem::kBarOff;
+    auto full_k = [&](int s) { return bar_base + 8u * s; };
+    auto full_v = [&](int s) { return bar_base + 8u * (kStages + s); };
+    auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+    const uint32_t merge_bar0 = bar_base + 8u * (3 * kStages);
+    const uint32_t merge_bar1 = merge_bar0 + 8u;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int32_t W = p.hdr[kHdrTotalTiles];
+    const int32_t R = p.hdr[kHdrNumRanges];
+    const int32_t P = p.page_size;
+    const int64_t max_len = (int64_t)p.bt_stride * P;
+    const bool cached = p.batch <= kSmemBatch;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_k(s), 1);
+            mbar_init(full_v(s), 1);
+            mbar_init(empty(s), kConsumerWarps);
+        }
+        mbar_init(merge_bar0, kConsumerWarps * 32);
+        mbar_init(merge_bar1, kConsumerWarps * 32);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (cached) {
+        for (int i = tid; i <= p.batch; i += kThreads) sm_prefix[i] = p.tiles_prefix[i];
+        for (int i = tid; i < p.batch; i += kThreads) {
+            int64_t n = p.seq_lens[i];
+            sm_len[i] = (int32_t)(n < 0 ? 0 : (n > max_len ? max_len : n));
+        }
+    }
+    __syncthreads();
+    const int32_t* prefix = cached ? sm_prefix : p.tiles_prefix;
+
+    if (warp == kConsumerWarps) {
+        // =========================================================== producer warp
+        uint32_t it = 0;                       // tiles issued so far
+        int32_t r = 0;
+        if (lane == 0) r = atomicAdd(p.hdr + kHdrClaim, 1);
+        r = __shfl_sync(0xffffffffu, r, 0);
+        bool ok = true;
+        const int pages_per_tile_shift = 6 - p.page_shift;      // log2(64 / P)
+        const uint32_t box_bytes = (uint32_t)P * kRowBytes;
+        while (ok && r < R) {
+            // claim the next range now; its latency hides behind this range's copies
+            int32_t r_next = 0;
+            if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
+            const int32_t x0 = (int32_t)(((int64_t)W * r) / R);
+            const int32_t x1 = (int32_t)(((int64_t)W * (r + 1)) / R);
+            int32_t x = x0;
+            while (ok && x < x1) {
+                const Segment sg = segment_at(prefix, p.batch, r, x0, x1, x);
+                x += sg.tile1 - sg.tile0;
+                int32_t n;
+                if (cached) n = sm_len[sg.b];
+                else { int64_t nn = p.seq_lens[sg.b]; n = (int32_t)(nn < 0 ? 0 : (nn > max_len ? max_len : nn)); }
+                const int32_t* table = p.block_table + (int64_t)sg.b * p.bt_stride;
+                const int32_t page_end = (min(sg.tile1 * kTile, n) + P - 1) >> p.page_shift;   // pages used by the segment
+                int32_t chunk_base = (sg.tile0 << pages_per_tile_shift);
+                // this lane's entry of the current 32-page chunk of the block table
+                int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
+                for (int32_t t = sg.tile0; ok && t < sg.tile1; ++t) {
+                    const int32_t first_page = t << pages_per_tile_shift;
+                    if (first_page >= chunk_base + 32) {
+                        chunk_base = first_page;
+                        pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
+                    }
+                    const int32_t n_valid = min(kTile, n - t * kTile);
+                    const int32_t npages = (n_valid + P - 1) >> p.page_shift;
+                    const int s = it % kStages;
+                    const uint32_t parity = (it / kStages) & 1u;
+                    // page ids of this tile, clamped into the pool
+                    int32_t my_page = __shfl_sync(0xffffffffu, pg, (first_page - chunk_base + (lane & 3)) & 31);
+                    bool bad = (lane < npages) && (my_page < 0 || my_page >= p.num_pages);
+                    if (__any_sync(0xffffffffu, bad)) {
+                        if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagBadPage);
+                        if (my_page < 0 || my_page >= p.num_pages) my_page = 0;
+                    }
+                    const int32_t page0 = __shfl_sync(0xffffffffu, my_page, 0);
+                    const int32_t page1 = __shfl_sync(0xffffffffu, my_page, 1);
+                    const int32_t page2 = __shfl_sync(0xffffffffu, my_page, 2);
+                    const int32_t page3 = __shfl_sync(0xffffffffu, my_page, 3);
+                    if (lane == 0) {
+                        ok = mbar_wait(empty(s), parity ^ 1u, abort_flag);
+                        if (ok) {
+                            StageMeta& m = meta[s];
+                            m.b = sg.b; m.g = sg.g; m.slot = sg.slot; m.n_valid = n_valid;
+                            m.first = (t == sg.tile0); m.last = (t == sg.tile1 - 1);
+                            const uint32_t kdst = smem_base + s * kStageBytes;
+                            const uint32_t vdst = kdst + kTileBytes;
+                            const bool with_q = (t == sg.tile0);
+                            mbar_arrive_expect_tx(full_k(s), npages * box_bytes + (with_q ? kQBytes : 0));
+                            if (with_q)
+                                bulk_load(vdst + kTileBytes, p.q + ((int64_t)sg.b * kHq + sg.g * kGroup) * kD,
+                                          kQBytes, full_k(s));
+                            const int32_t pages[4] = {page0, page1, page2, page3};
+                            #pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                if (i < npages)
+                                    tma_load_tile(kdst + i * box_bytes, &map_k, (pages[i] * kHkv + sg.g) * P, full_k(s));
+                            mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
+                            #pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                if (i < npages)
+                                    tma_load_tile(vdst + i * box_bytes, &map_v, (pages[i] * kHkv + sg.g) * P, full_v(s));
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (ok) ++it;
+                }
+            }
+            r = __shfl_sync(0xffffffffu, r_next, 0);
+        }
+        if (lane == 0) {
+            if (ok) {
+                // tell the consumers that there is no more work
+                const int s = it % kStages;
+                const uint32_t parity = (it / kStages) & 1u;
+                ok = mbar_wait(empty(s), parity ^ 1u, abort_flag);
+                if (ok) {
+                    meta[s].n_valid = 0;
+                    mbar_arrive(full_k(s));
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                // let the copies still in flight land before the CTA's shared memory is released
+                const uint32_t lo = it > (uint32_t)kStages ? it - kStages : 0u;
+                for (uint32_t j = lo; j < it; ++j) {
+                    volatile int32_t never = 0;
+                    mbar_wait(full_k(j % kStages), (j / kStages) & 1u, &never);
+                    mbar_wait(full_v(j % kStages), (j / kStages) & 1u, &never);
+                }
+            }
+        }
+        return;
+    }
+
+    // =============================================================== consumer warps
+    const int quad = lane & 3;           // selects this thread's two heads: 2*quad, 2*quad + 1
+    const int qrow = lane >> 2;          // row inside an 8-row fragment block
+    const float ninf = -INFINITY;
+    // per-lane pieces of the swizzled tile addresses (see the layout note at tma_load_tile):
+    // a 64-token tile is 64/P boxes; a box is [2 halves][P rows][128 B], 16-byte chunks of a
+    // row XOR-ed with (row & 7)
+    const int tok0 = warp * 16;                                   // this warp's first token in the tile
+    const uint32_t box_off = (uint32_t)(tok0 >> p.page_shift) * (uint32_t)P * kRowBytes;
+    const uint32_t half_stride = (uint32_t)P * 128u;
+    const int rb0 = tok0 & (P - 1);
+    // K fragments (non-transposed): matrices (rows 0-7 | 8-15) x (k 0-7 | 8-15)
+    const int k_row = rb0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const uint32_t k_row_off = box_off + (uint32_t)k_row * 128u;
+    const int k_sel = lane >> 4;                                  // 16-byte chunk inside the 32-byte k-step
+    // V fragments (transposed): matrices (tok 0-7 | 8-15) x (d 0-7 | 8-15), ordered for A = V^T
+    const int v_row = rb0 + (lane & 7) + (lane >> 4) * 8;
+    const uint32_t v_row_off = box_off + (uint32_t)v_row * 128u;
+    const int v_sel = (lane >> 3) & 1;
+
+    uint32_t qf[8][2];
+    float m0 = ninf, m1 = ninf, l0 = 0.f, l1 = 0.f;
+    float o[8][4];
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) { qf[i][0] = qf[i][1] = 0u; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    uint32_t merges = 0;
+
+    for (uint32_t it = 0;; ++it) {
+        const int s = it % kStages;
+        const uint32_t parity = (it / kStages) & 1u;
+        if (!mbar_wait(full_k(s), parity, abort_flag)) {
+            *abort_flag = 1;
+            if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+            return;
+        }
+        const StageMeta mt = meta[s];
+        if (mt.n_valid == 0) return;
+        const uint32_t kbase = smem_base + s * kStageBytes;
+        const uint32_t vbase = kbase + kTileBytes;
+        if (mt.first) {
+            const uint32_t* qs = reinterpret_cast<const uint32_t*>(smem + s * kStageBytes + 2 * kTileBytes);
+            #pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qf[ks][0] = qs[qrow * (kD / 2) + ks * 8 + quad];
+                qf[ks][1] = qs[qrow * (kD / 2) + ks * 8 + quad + 4];
+            }
+            m0 = m1 = ninf; l0 = l1 = 0.f;
+            #pragma unroll
+            for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        }
+        const int valid = mt.n_valid - tok0;          // valid tokens among this warp's 16
+        if (valid > 0) {
+            // ---- S^T = K . Q^T  (two accumulator chains to shorten the dependency)
+            float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+            #pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const int chunk = ks * 2 + k_sel;
+                const uint32_t addr = kbase + k_row_off + (uint32_t)(chunk >> 3) * half_stride +
+                                      (uint32_t)(((chunk & 7) ^ (k_row & 7)) << 4);
+                uint32_t a[4];
+                ldmatrix_x4(addr, a);
+                if (ks & 1) mma_bf16(sb, a, qf[ks][0], qf[ks][1]);
+                else mma_bf16(sa, a, qf[ks][0], qf[ks][1]);
+            }
+            // scores of tokens (qrow, qrow + 8) for heads (2 quad, 2 quad + 1), base-2 domain
+            float s00 = (sa[0] + sb[0]) * p.scale_log2e, s01 = (sa[1] + sb[1]) * p.scale_log2e;
+            float s10 = (sa[2] + sb[2]) * p.scale_log2e, s11 = (sa[3] + sb[3]) * p.scale_log2e;
+            if (qrow >= valid) { s00 = ninf; s01 = ninf; }
+            if (qrow + 8 >= valid) { s10 = ninf; s11 = ninf; }
+            float bm0 = fmaxf(s00, s10), bm1 = fmaxf(s01, s11);
+            #pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
+                bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
+            }
+            const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);
+            if (__any_sync(0xffffffffu, (n0 != m0) || (n1 != m1))) {
+                const float a0 = fast_exp2(m0 - n0), a1 = fast_exp2(m1 - n1);   // exp2(-inf) = 0 on first use
+                l0 *= a0; l1 *= a1;
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) { o[i][0] *= a0; o[i][1] *= a1; o[i][2] *= a0; o[i][3] *= a1; }
+                m0 = n0; m1 = n1;
+            }
+            const float p00 = fast_exp2(s00 - m0), p01 = fast_exp2(s01 - m1);
+            const float p10 = fast_exp2(s10 - m0), p11 = fast_exp2(s11 - m1);
+            l0 += p00 + p10;
+            l1 += p01 + p11;
+            // P^T as the B operand: transpose the two 8x8 (token x head) blocks in registers
+            const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01));
+            const uint32_t pb1 = movmatrix_trans(pack_bf16(p10, p11));
+
+            if (!mbar_wait(full_v(s), parity, abort_flag)) {
+                *abort_flag = 1;
+                if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                return;
+            }
+            if (valid < 16) {
+                // rows past the end of the sequence may hold anything (NaN included) and a zero
+                // probability does not silence them inside an MMA: clear them first
+                for (int i = lane; i < (16 - valid) * 16; i += 32) {
+                    const int row = rb0 + valid + (i >> 4);
+                    const int c = i & 15;
+                    const uint32_t addr = vbase + box_off + (uint32_t)(c >> 3) * half_stride + (uint32_t)row * 128u +
+                                          (uint32_t)((c & 7) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+            }
+            // ---- O^T += V^T . P^T
+            #pragma unroll
+            for (int db = 0; db < 8; ++db) {
+                const int chunk = db * 2 + v_sel;
+                const uint32_t addr = vbase + v_row_off + (uint32_t)(chunk >> 3) * half_stride +
+                                      (uint32_t)(((chunk & 7) ^ (v_row & 7)) << 4);
+                uint32_t a[4];
+                ldmatrix_x4_trans(addr, a);
+                mma_bf16(o[db], a, pb0, pb1);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty(s));
+
+        if (mt.last) {
+            // ---- merge the four warps' states and write the segment's result
+            #pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+            }
+            float* mo = merge_o + warp * (kGroup * kMergeStride);
+            #pragma unroll
+            for (int db = 0; db < 8; ++db) {
+                const int d = db * 16 + qrow;
+                mo[(2 * quad) * kMergeStride + d] = o[db][0];
+                mo[(2 * quad + 1) * kMergeStride + d] = o[db][1];
+                mo[(2 * quad) * kMergeStride + d + 8] = o[db][2];
+                mo[(2 * quad + 1) * kMergeStride + d + 8] = o[db][3];
+            }
+            if (qrow == 0) {
+                float* ml = merge_ml + (warp * kGroup + 2 * quad) * 2;
+                ml[0] = m0; ml[1] = l0; ml[2] = m1; ml[3] = l1;
+            }
+            mbar_arrive(merge_bar0);
+            if (!mbar_wait(merge_bar0, merges & 1u, abort_flag)) {
+                *abort_flag = 1;
+                if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                return;
+            }
+            const int d = tid;                        // 128 consumer threads = 128 dims
+            #pragma unroll
+            for (int h = 0; h < kGroup; ++h) {
+                float M = ninf;
+                #pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_ml[(w * kGroup + h) * 2]);
+                float L = 0.f, acc = 0.f;
+                #pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float wt = fast_exp2(merge_ml[(w * kGroup + h) * 2] - M);
+                    L = fmaf(merge_ml[(w * kGroup + h) * 2 + 1], wt, L);
+                    acc = fmaf(merge_o[(w * kGroup + h) * kMergeStride + d], wt, acc);
+                }
+                const float res = acc / L;
+                const float lse2 = M + log2f(L);
+                if (mt.slot < 0) {
+                    const int64_t row = (int64_t)mt.b * kHq + mt.g * kGroup + h;
+                    p.out[row * kD + d] = __float2bfloat16_rn(res);
+                    if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
+                } else {
+                    const int64_t row = (int64_t)mt.slot * kGroup + h;
+                    p.part_o[row * kD + d] = res;
+                    if (d == 0) p.part_lse[row] = lse2;
+                }
+            }
+            mbar_arrive(merge_bar1);
+            if (!mbar_wait(merge_bar1, merges & 1u, abort_flag)) {
+                *abort_flag = 1;
+                if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                return;
+            }
+            ++merges;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            sym = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(sym);
+    }();
+    return fn;
+}
+
+// A pool [num_pages][8][P][128] bf16 seen as {64 elements, rows, 2 halves}: element stride 2 B,
+// row stride 256 B, half stride 128 B.  A box {64, P, 2} is one (page, head) chunk and lands in
+// shared memory as [half][row][128 B] with the 128-byte swizzle.
+bool make_pool_map(CUtensorMap* map, const void* pool, int32_t num_pages, int32_t P) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * kHkv * P, 2};
+    const cuuint64_t strides[2] = {256, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)P, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    } else if (dev >= 64) {
+        e = cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+    }
+    CUtensorMap map_k, map_v;
+    if (!make_pool_map(&map_k, p.k_pages, p.num_pages, p.page_size) ||
+        !make_pool_map(&map_v, p.v_pages, p.num_pages, p.page_size))
+        return cudaErrorInvalidValue;
+    partial_mma_kernel<<<p.grid_ctas, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
+    return cudaGetLastError();
+}
+
+}  // namespace concur

@@ -1,0 +1,94 @@
+// Plan kernel: per-sequence tile counts, their prefix sums, and the split-KV ranges.
+//
+// The KV cache of the batch is seen as one flat list of W = Hkv * sum_b ceil(len_b / 64)
+// tiles (sequence-major, then KV head, then position).  The plan cuts [0, W) into R
+// ranges of equal size (to within one tile).  CTAs of the partial kernel claim ranges
+// one after another, so ragged context lengths balance over the SMs no matter how the
+// lengths are distributed; a sequence is split exactly where a range boundary falls
+// inside one of its (sequence, KV head) units.
+#include "common.cuh"
+
+namespace concur {
+
+constexpr int kPlanThreads = 1024;
+
+__global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
+    __shared__ int32_t warp_sums[kPlanThreads / 32];
+    __shared__ int32_t carry_s;
+    __shared__ int32_t ranges_s;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) { carry_s = 0; p.tiles_prefix[0] = 0; }
+    __syncthreads();
+
+    const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
+    uint32_t flags = 0;
+    for (int base = 0; base < p.batch; base += kPlanThreads) {
+        int b = base + tid;
+        int32_t tiles = 0;
+        if (b < p.batch) {
+            int64_t len = p.seq_lens[b];
+            if (len < 0) { len = 0; flags |= kFlagBadLen; }
+            if (len > max_len) { len = max_len; flags |= kFlagBadLen; }
+            tiles = (int32_t)((len + kTile - 1) / kTile);
+        }
+        // inclusive scan over the block
+        int32_t v = tiles;
+        #pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int32_t n = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += n;
+        }
+        if (lane == 31) warp_sums[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t w = warp_sums[lane];
+            #pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int32_t n = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += n;
+            }
+            warp_sums[lane] = w;
+        }
+        __syncthreads();
+        int32_t incl = v + (warp ? warp_sums[warp - 1] : 0) + carry_s;
+        if (b < p.batch) p.tiles_prefix[b + 1] = incl;
+        __syncthreads();
+        if (tid == kPlanThreads - 1) carry_s = incl;
+        __syncthreads();
+    }
+    if (flags) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), flags);
+
+    if (tid == 0) {
+        const int32_t W = kHkv * carry_s;
+        int32_t R;
+        if (p.forced_ranges > 0) {
+            R = p.forced_ranges;
+        } else {
+            // as many ranges as keeps every CTA supplied `ranges_per_cta` times over,
+            // but none shorter than `min_range_tiles`
+            R = W / p.min_range_tiles;
+            int32_t cap = p.grid_ctas * p.ranges_per_cta;
+            if (R > cap) R = cap;
+        }
+        if (R > p.max_ranges) R = p.max_ranges;
+        if (R > W) R = W;
+        if (R < 1 && W > 0) R = 1;
+        p.hdr[kHdrTotalTiles] = W;
+        p.hdr[kHdrNumRanges] = R;
+        p.hdr[kHdrClaim] = 0;
+        ranges_s = R;
+    }
+    __syncthreads();
+    const int32_t R = ranges_s;
+    const int64_t W = (int64_t)kHkv * carry_s;
+    for (int r = tid; r <= R; r += kPlanThreads)
+        p.range_start[r] = (R > 0) ? (int32_t)((W * r) / R) : 0;
+}
+
+cudaError_t launch_plan(const DecodeParams& p, cudaStream_t stream) {
+    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace concur

@@ -1,0 +1,62 @@
+"""Test-side helpers: the oracle run over many sequences with a thread pool (the oracle
+itself stays single-threaded; ctypes releases the GIL), and the parity criteria."""
+from __future__ import annotations
+
+import os
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import torch
+
+import oracle
+
+# tolerance of the bf16 output and fp32 lse against the fp64 oracle
+OUT_ATOL, OUT_RTOL = 4e-3, 1.6e-2
+LSE_ATOL = 1e-3
+REL_RMS_MAX = 5e-3          # stricter internal gate on the whole output
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_sequences(w, seqs=None, threads=None):
+    """Oracle for the given sequences of a host-resident workload.  Returns
+    (out [len(seqs)][Hq][D] f64, lse [len(seqs)][Hq] f64)."""
+    seqs = list(range(w.spec.batch)) if seqs is None else list(seqs)
+    qb = oracle._u16(w.q); kb = oracle._u16(w.k_pages); vb = oracle._u16(w.v_pages)
+    tb = oracle._i32(w.block_table); lb = oracle._i32(w.seq_lens)
+
+    def one(b):
+        o, l = oracle.decode_attn(qb, kb, vb, tb, lb, w.scale, seqs=(b, b + 1))
+        return o[b], l[b]
+
+    with ThreadPoolExecutor(max_workers=threads or host_cores()) as ex:
+        res = list(ex.map(one, seqs))
+    if not res:
+        return np.zeros((0, w.spec.num_q_heads, w.spec.head_dim)), np.zeros((0, w.spec.num_q_heads))
+    return np.stack([r[0] for r in res]), np.stack([r[1] for r in res])
+
+
+def assert_parity(out_gpu, lse_gpu, ref_out, ref_lse, what=""):
+    """out_gpu bf16 / lse_gpu fp32 torch tensors (any device) against fp64 numpy references."""
+    og = out_gpu.detach().cpu().to(torch.float64).numpy()
+    lg = lse_gpu.detach().cpu().to(torch.float64).numpy()
+    assert og.shape == ref_out.shape and lg.shape == ref_lse.shape, what
+    assert np.isfinite(og).all(), f"{what}: non-finite output"
+    err = np.abs(og - ref_out)
+    bound = OUT_ATOL + OUT_RTOL * np.abs(ref_out)
+    worst = np.unravel_index(np.argmax(err - bound), err.shape)
+    assert (err <= bound).all(), f"{what}: out[{worst}] = {og[worst]} vs {ref_out[worst]}"
+    empty = np.isneginf(ref_lse)
+    assert np.array_equal(np.isneginf(lg), empty), f"{what}: lse -inf pattern"
+    lerr = np.abs(lg[~empty] - ref_lse[~empty])
+    assert lerr.size == 0 or lerr.max() <= LSE_ATOL, f"{what}: lse error {lerr.max()}"
+    den = np.sqrt(np.mean(ref_out ** 2))
+    rel_rms = float(np.sqrt(np.mean(err ** 2)) / den) if den > 0 else 0.0
+    assert rel_rms <= REL_RMS_MAX, f"{what}: relative RMS error {rel_rms}"
+    return {"max_abs": float(err.max()) if err.size else 0.0, "rel_rms": rel_rms,
+            "lse_max_abs": float(lerr.max()) if lerr.size else 0.0}
