@@ -56,6 +56,8 @@ SPECS = {
     "cfg1_b1_ctx512_p16": Spec("cfg1_b1_ctx512_p16", 1, 16, ("const", 512), permute_pages=False, seed=73561),
     "cfg2_b16_u1k_8k_p16": Spec("cfg2_b16_u1k_8k_p16", 16, 16, ("uniform", 1024, 8192), seed=73562),
     "cfg3_b64_ctx16384_p64": Spec("cfg3_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563),
+    # a quarter of cfg3 (same lengths, page size and values): small enough for profiler captures
+    "cfg3q_b16_ctx16384_p64": Spec("cfg3q_b16_ctx16384_p64", 16, 64, ("const", 16384), q_std=0.5, seed=73563),
     "cfg4_b256_logu2k_32k_p64": Spec("cfg4_b256_logu2k_32k_p64", 256, 64, ("loguniform", 2048, 32768), seed=73564),
     "cfg5_b32_skew128k_p64": Spec("cfg5_b32_skew128k_p64", 32, 64, ("skew", 131072, 256, 4096),
                                   k_outlier_prob=0.01, seed=73565),
