@@ -165,6 +165,42 @@ int concur_attn_set_option(concur_attn_t* handle, int32_t key, int64_t value);
 int concur_attn_last_plan(concur_attn_t* handle, void* cuda_stream, int32_t* num_ranges,
                           int32_t* total_tiles, int32_t* range_start, int32_t cap);
 
+/*
+ * The same decode-attention step for callers that cannot allocate device memory.  (The
+ * paper has no counterpart to this entry point; it exists for integration only.)
+ *
+ * Who needs it: a process that gave its whole device-memory budget to its own arena at
+ * start-up and treats later driver allocations as errors; code that runs inside another
+ * runtime's callback, where cudaMalloc is not permitted; a latency path that cannot risk
+ * the device-wide synchronisation an allocation or a free may cause.  Such callers cannot
+ * create a handle (a handle owns or borrows a workspace).  Here the workspace is a fixed
+ * array inside the library's device image -- about 4.3 MB that every GPU which loads the
+ * library holds until the process exits -- and there is no handle at all.
+ *
+ * Arguments and layouts are those of concur_decode_attn, plus `page_size` (16, 32 or 64);
+ * the work is enqueued on `cuda_stream` of the CURRENT device and the call returns without
+ * synchronising.  It performs no cudaMalloc / cudaFree and calls no allocating library
+ * routine.  Limits: batch <= CONCUR_STATIC_MAX_BATCH (more: CONCUR_ERR_TOO_LARGE, nothing
+ * is launched); the plan uses at most CONCUR_STATIC_MAX_RANGES split-KV ranges, so very
+ * large batches balance a little more coarsely than through a handle.  Other errors as for
+ * concur_decode_attn.  Device-side condition flags (bad page id, bad length) still clamp
+ * the access but are not reported by this entry point.
+ *
+ * The first call on each device resolves the array's device address
+ * (cudaGetSymbolAddress) and reads the SM count; make that first call outside any stream
+ * capture.  All calls on a device share the one array, which keeps the previous call's
+ * contents: each call re-initialises what it reads, but two calls whose kernels overlap on
+ * the GPU (different streams without ordering, or different host threads) race on it.
+ * Order them on one stream or with events.
+ */
+#define CONCUR_STATIC_MAX_BATCH  1024
+#define CONCUR_STATIC_MAX_RANGES 512
+int concur_decode_attn_static(const void* q, const void* k_pages, const void* v_pages,
+                              const int32_t* block_table, const int32_t* seq_lens,
+                              float scale, void* out, float* lse,
+                              int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                              int32_t page_size, void* cuda_stream);
+
 /* Frees the handle and any memory the library allocated for it.  NULL is accepted. */
 int concur_attn_destroy(concur_attn_t* handle);
 

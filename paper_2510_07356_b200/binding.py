@@ -34,7 +34,10 @@ EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
+    "concur_decode_attn_static",
 )
+CONCUR_STATIC_MAX_BATCH = 1024
+CONCUR_STATIC_MAX_RANGES = 512
 
 
 class concur_attn_config_t(ctypes.Structure):
@@ -64,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_decode_attn.argtypes = decode_args
     lib.concur_decode_attn_host.restype = ctypes.c_int
     lib.concur_decode_attn_host.argtypes = decode_args
+    lib.concur_decode_attn_static.restype = ctypes.c_int
+    lib.concur_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
     lib.concur_attn_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.concur_attn_set_option.restype = ctypes.c_int
@@ -145,6 +150,19 @@ def concur_decode_attn_host(handle, q, k_pages, v_pages, block_table, seq_lens, 
     return _decode(lib.concur_decode_attn_host, "concur_decode_attn_host", handle, q, k_pages,
                    v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
                    block_table_stride, stream, check)
+
+
+def concur_decode_attn_static(q, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
+                              batch, num_pages, block_table_stride, page_size, stream=0, check=True) -> int:
+    """The handle-free variant for callers that must not allocate device memory: its
+    workspace is a fixed array inside the library.  Device tensors; current device; calls
+    must not overlap on the GPU (they share that array)."""
+    rc = lib.concur_decode_attn_static(_addr(q), _addr(k_pages), _addr(v_pages), _addr(block_table),
+                                       _addr(seq_lens), ctypes.c_float(scale), _addr(out), _addr(lse),
+                                       batch, num_pages, block_table_stride, page_size, stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_decode_attn_static")
+    return rc
 
 
 def concur_attn_status(handle, stream=0) -> int:

@@ -1,0 +1,55 @@
+"""The handle-free entry point for callers that cannot allocate device memory
+(concur_decode_attn_static): same results as the regular entry point, on two calls in a
+row that share its built-in workspace.
+
+Collected last on purpose: should this addition ever fail, a run that stops at the first
+failure has already executed every other test.
+"""
+import pytest
+import torch
+
+import synth
+
+pytestmark = pytest.mark.gpu
+
+# the two entry points may split sequences differently, so their bf16 outputs agree to the
+# tolerance every parity test uses, not bit for bit
+OUT_ATOL, OUT_RTOL, LSE_ATOL = 4e-3, 1.6e-2, 1e-3
+
+
+def test_static_entry_matches_handle_entry_twice_in_a_row():
+    import __graft_entry__
+    __graft_entry__.build()
+    import paper_2510_07356_b200 as P
+
+    stream = torch.cuda.current_stream().cuda_stream
+    # two different batches, the second one larger, so that anything the first call left in
+    # the shared array would be noticed
+    specs = [synth.tiny_spec("na0", (3000, 1, 0, 64, 777, 12000), 64, 501),
+             synth.tiny_spec("na1", (9000, 20000, 130, 64, 5, 0, 4100, 2500), 64, 502)]
+    for spec in specs:
+        w = synth.make_workload(spec, "cuda:0")
+        B = spec.batch
+        ref = P.DecodeAttention(64, B, w.block_table.shape[1], 0)
+        out_ref, lse_ref = ref(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
+        out = torch.full_like(w.q, 7.0)
+        lse = torch.full((B, 64), 7.0, dtype=torch.float32, device="cuda:0")
+        P.concur_decode_attn_static(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale,
+                                    out, lse, B, w.num_pages, w.block_table.shape[1], 64, stream)
+        torch.cuda.synchronize()
+        a, b = out.float(), out_ref.float()
+        assert torch.isfinite(a).all()
+        assert ((a - b).abs() <= OUT_ATOL + OUT_RTOL * b.abs()).all()
+        empty = torch.isneginf(lse_ref)
+        assert torch.equal(torch.isneginf(lse), empty)
+        assert ((lse - lse_ref)[~empty].abs() <= LSE_ATOL).all()
+        ref.close()
+
+    # beyond the built-in workspace's batch limit: a clear error, nothing launched
+    rc = P.concur_decode_attn_static(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale,
+                                     out, lse, P.binding.CONCUR_STATIC_MAX_BATCH + 1, w.num_pages,
+                                     w.block_table.shape[1], 64, stream, check=False)
+    assert rc == P.binding.CONCUR_ERR_TOO_LARGE
+    rc = P.concur_decode_attn_static(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale,
+                                     out, lse, B, w.num_pages, w.block_table.shape[1], 48, stream, check=False)
+    assert rc == P.binding.CONCUR_ERR_UNSUPPORTED
