@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--ranges-per-cta", type=int, default=0)
     ap.add_argument("--min-range-tiles", type=int, default=0)
     ap.add_argument("--num-ranges", type=int, default=0)
+    ap.add_argument("--fuse-combine", type=int, default=-1)
+    ap.add_argument("--claim-ahead", type=int, default=-1)
     return ap.parse_args()
 
 
@@ -253,6 +255,10 @@ def main():
     attn.set_option(P.CONCUR_OPT_RANGES_PER_CTA, args.ranges_per_cta)
     attn.set_option(P.CONCUR_OPT_MIN_RANGE_TILES, args.min_range_tiles)
     attn.set_option(P.CONCUR_OPT_NUM_RANGES, args.num_ranges)
+    if args.fuse_combine >= 0:
+        attn.set_option(P.CONCUR_OPT_FUSE_COMBINE, args.fuse_combine)
+    if args.claim_ahead >= 0:
+        attn.set_option(P.CONCUR_OPT_CLAIM_AHEAD, args.claim_ahead)
     out = torch.empty_like(w.q)
     lse = torch.empty((spec.batch, spec.num_q_heads), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream(dev)
@@ -276,13 +282,8 @@ def main():
     barrier()
     assert attn.status() == 0, "device-side flags set during warm-up"
 
-    # ---- timed region: K whole steps; events around each step and around its partial kernel
+    # ---- timed region: K whole steps, one event pair around the region
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    for row in ev:                       # materialise the cudaEvent_t handles
-        for e in row:
-            e.record(stream)
-    torch.cuda.synchronize(dev)
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
@@ -291,24 +292,42 @@ def main():
     if rank == 0:
         sampler.start()
         time.sleep(0.2)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K + 1)]
+    for row in ev:                       # materialise the cudaEvent_t handles
+        for e in row:
+            e.record(stream)
     barrier()
     t_mark0 = time.time()
+    if flush_buf is None:
+        ev[K][0].record(stream)
+        for i in range(K):
+            step()
+        ev[K][1].record(stream)
+        barrier()
+        ms_per_step = ev[K][0].elapsed_time(ev[K][1]) / K
+        step_ms = [ms_per_step]
+    else:                                # small inputs: L2 is flushed before every step, steps timed one by one
+        for i in range(K):
+            flush_buf.zero_()
+            ev[i][0].record(stream)
+            step()
+            ev[i][1].record(stream)
+        barrier()
+        step_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
+        ms_per_step = sum(step_ms) / K
+    # ---- the same K steps again with events recorded by the library around its partial kernel
     for i in range(K):
         if flush_buf is not None:
             flush_buf.zero_()
-        attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, ev[i][1].cuda_event)
-        attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, ev[i][2].cuda_event)
-        ev[i][0].record(stream)
+        attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, ev[i][0].cuda_event)
+        attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, ev[i][1].cuda_event)
         step()
-        ev[i][3].record(stream)
     barrier()
     t_mark1 = time.time()
     clocks = sampler.stop(t_mark0, t_mark1) if rank == 0 else None
     attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, 0)
     attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, 0)
-    step_ms = [ev[i][0].elapsed_time(ev[i][3]) for i in range(K)]
-    part_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)]
-    ms_per_step = sum(step_ms) / K
+    part_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
     part_ms_avg = sum(part_ms) / K
     if world > 1:
         t = torch.tensor([ms_per_step, part_ms_avg], dtype=torch.float64, device=dev)
@@ -373,7 +392,7 @@ def main():
                      "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "partial", "ms": part_ms_avg,
                      "ms_min": min(part_ms)},
         "step_ms_min": min(step_ms),
-        "e2e": e2e, "gpu_launches": 3 * K, "clocks": clocks, "device_flags": flags,
+        "e2e": e2e, "gpu_launches": (2 if args.kernel == 0 else 3) * K, "clocks": clocks, "device_flags": flags,
     }
     if not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)

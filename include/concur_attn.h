@@ -66,12 +66,16 @@ typedef enum {
 #define CONCUR_OPT_KERNEL      1    /* 0 = tensor-core partial kernel (default), 1 = scalar-FMA kernel */
 #define CONCUR_OPT_NUM_RANGES  2    /* force the number of split-KV ranges; 0 = heuristic              */
 #define CONCUR_OPT_GRID_CTAS   3    /* force the partial kernel's grid size; 0 = one wave of the GPU    */
-#define CONCUR_OPT_RANGES_PER_CTA 4 /* heuristic's target ranges per CTA; 0 = built-in default          */
-#define CONCUR_OPT_MIN_RANGE_TILES 5/* heuristic's smallest range, in 64-token tiles; 0 = default       */
+#define CONCUR_OPT_RANGES_PER_CTA 4 /* heuristic's target ranges per CTA; 0 = built-in default (1)      */
+#define CONCUR_OPT_MIN_RANGE_TILES 5/* heuristic's smallest range, in 64-token tiles; 0 = default (2)   */
 #define CONCUR_OPT_EVENT_BEFORE_PARTIAL 6 /* a cudaEvent_t (as an integer) recorded on the call's stream
                                              just before the partial kernel; 0 = none.  For timing
                                              that kernel alone; the event stays the caller's.          */
 #define CONCUR_OPT_EVENT_AFTER_PARTIAL  7 /* likewise, just after the partial kernel                    */
+#define CONCUR_OPT_FUSE_COMBINE 8   /* tensor-core kernel: 1 (default) = the CTA that finishes a unit's last
+                                       partial merges the unit in-kernel; 0 = separate combine kernel   */
+#define CONCUR_OPT_CLAIM_AHEAD  9   /* tiles before a range's end at which a CTA claims its next range
+                                       (default: at the range's first tile)                              */
 
 typedef struct concur_attn concur_attn_t;   /* opaque; owns its workspace and nothing else */
 

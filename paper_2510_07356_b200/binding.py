@@ -29,6 +29,8 @@ CONCUR_OPT_RANGES_PER_CTA = 4
 CONCUR_OPT_MIN_RANGE_TILES = 5
 CONCUR_OPT_EVENT_BEFORE_PARTIAL = 6
 CONCUR_OPT_EVENT_AFTER_PARTIAL = 7
+CONCUR_OPT_FUSE_COMBINE = 8
+CONCUR_OPT_CLAIM_AHEAD = 9
 
 EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",

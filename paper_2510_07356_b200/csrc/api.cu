@@ -17,7 +17,7 @@ constexpr size_t kAlign = 256;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct WorkspaceLayout {
-    size_t hdr, prefix, range_start, part_lse, part_o, total;
+    size_t hdr, prefix, range_start, unit_done, part_lse, part_o, total;
 };
 
 WorkspaceLayout layout_for(int32_t max_batch) {
@@ -26,6 +26,7 @@ WorkspaceLayout layout_for(int32_t max_batch) {
     w.hdr = at;          at += align_up(kHdrWords * sizeof(int32_t));
     w.prefix = at;       at += align_up(((size_t)max_batch + 1) * sizeof(int32_t));
     w.range_start = at;  at += align_up(((size_t)kMaxRanges + 1) * sizeof(int32_t));
+    w.unit_done = at;    at += align_up((size_t)max_batch * kHkv * sizeof(int32_t));
     w.part_lse = at;     at += align_up((size_t)2 * kMaxRanges * kGroup * sizeof(float));
     w.part_o = at;       at += align_up((size_t)2 * kMaxRanges * kGroup * kD * sizeof(float));
     w.total = at;
@@ -80,6 +81,8 @@ struct concur_attn {
     int32_t grid_ctas = 0;
     int32_t ranges_per_cta = 0;
     int32_t min_range_tiles = 0;
+    int32_t fuse_combine = 1;
+    int32_t claim_ahead = 1 << 20;
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;
     Staging st_q, st_k, st_v, st_bt, st_len, st_out, st_lse;
 };
@@ -146,12 +149,15 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     const int per_sm = h->kernel == 1 ? partial_scalar_ctas_per_sm() : 1;
     p.grid_ctas = h->grid_ctas > 0 ? h->grid_ctas : h->sm_count * per_sm;
     p.forced_ranges = h->forced_ranges;
-    p.ranges_per_cta = h->ranges_per_cta > 0 ? h->ranges_per_cta : 16;
+    p.ranges_per_cta = h->ranges_per_cta > 0 ? h->ranges_per_cta : 1;
     p.min_range_tiles = h->min_range_tiles > 0 ? h->min_range_tiles : 2;
     p.max_ranges = kMaxRanges;
+    p.fuse_combine = h->fuse_combine;
+    p.claim_ahead = h->claim_ahead;
     p.hdr = reinterpret_cast<int32_t*>(h->ws + h->lay.hdr);
     p.tiles_prefix = reinterpret_cast<int32_t*>(h->ws + h->lay.prefix);
     p.range_start = reinterpret_cast<int32_t*>(h->ws + h->lay.range_start);
+    p.unit_done = reinterpret_cast<int32_t*>(h->ws + h->lay.unit_done);
     p.part_lse = reinterpret_cast<float*>(h->ws + h->lay.part_lse);
     p.part_o = reinterpret_cast<float*>(h->ws + h->lay.part_o);
     return CONCUR_OK;
@@ -179,7 +185,9 @@ static int enqueue(concur_attn_t* h, const DecodeParams& p, cudaStream_t stream)
     cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream);
     if (e != cudaSuccess) return CONCUR_ERR_CUDA;
     if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
-    if (launch_combine(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    // the tensor-core kernel merges split units itself; the scalar kernel leaves that to the
+    // combine kernel
+    if ((h->kernel == 1 || !h->fuse_combine) && launch_combine(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     return CONCUR_OK;
 }
 
@@ -282,6 +290,12 @@ int concur_attn_set_option(concur_attn_t* h, int32_t key, int64_t value) {
         case CONCUR_OPT_MIN_RANGE_TILES:
             if (value > (1 << 20)) return CONCUR_ERR_INVALID_ARG;
             h->min_range_tiles = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_FUSE_COMBINE:
+            if (value > 1) return CONCUR_ERR_INVALID_ARG;
+            h->fuse_combine = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_CLAIM_AHEAD:
+            if (value > (1 << 20)) return CONCUR_ERR_INVALID_ARG;
+            h->claim_ahead = (int32_t)value; return CONCUR_OK;
         case CONCUR_OPT_EVENT_BEFORE_PARTIAL:
             h->ev_before = reinterpret_cast<cudaEvent_t>(static_cast<uintptr_t>(value)); return CONCUR_OK;
         case CONCUR_OPT_EVENT_AFTER_PARTIAL:

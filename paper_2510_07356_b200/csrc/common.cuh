@@ -25,6 +25,7 @@ enum HeaderWord : int {
     kHdrNumRanges = 1,    // R: ranges the flat tile index space [0, W) is cut into
     kHdrClaim = 2,        // next range to hand out (atomic)
     kHdrStatus = 3,       // sticky CONCUR_FLAG_* bits
+    kHdrWaitSite = 4,     // which wait gave up first (diagnostic; 0 = none)
     kHdrWords = 64
 };
 
@@ -49,13 +50,29 @@ struct DecodeParams {
     int32_t ranges_per_cta;
     int32_t min_range_tiles;
     int32_t max_ranges;       // capacity of range_start / partial slots
+    int32_t fuse_combine;     // tensor-core kernel: 1 = the last partial of a unit merges it in-kernel
+    int32_t claim_ahead;      // tiles before a range's end at which the next range is claimed
     // workspace
     int32_t* hdr;             // [kHdrWords]
     int32_t* tiles_prefix;    // [batch + 1] exclusive prefix of per-sequence tile counts
     int32_t* range_start;     // [R + 1] boundaries in flat tile space
     float* part_o;            // [2 * max_ranges][kGroup][kD] normalised partial outputs
     float* part_lse;          // [2 * max_ranges][kGroup]     base-2 log-sum-exp of each partial
+    int32_t* unit_done;       // [batch * kHkv] partial segments finished per (sequence, KV head) unit
 };
+
+// First flat tile of range r when [0, W) is cut into R ranges of equal size.
+__device__ __forceinline__ int32_t range_begin(int32_t W, int32_t R, int32_t r) {
+    return (int32_t)(((int64_t)W * r) / R);
+}
+
+// The range that contains flat tile x (0 <= x < W), by arithmetic alone.
+__device__ __forceinline__ int32_t range_of(int32_t W, int32_t R, int32_t x) {
+    int32_t r = (int32_t)(((int64_t)x * R) / W);
+    while (r + 1 < R && range_begin(W, R, r + 1) <= x) ++r;
+    while (r > 0 && range_begin(W, R, r) > x) --r;
+    return r;
+}
 
 // The flat tile space lists, for sequence b = 0.., KV head g = 0..7, that unit's tiles:
 // unit (b, g) occupies [kHkv * prefix[b] + g * tiles_b, ... + tiles_b).

@@ -15,7 +15,8 @@
 // transposes.  When a segment (a run of tiles of one (sequence, KV head) unit inside a
 // range of the plan) ends, the four warps' states are merged through shared memory and
 // written either straight to out/lse (the segment was the whole unit) or to a partial
-// slot for the combine kernel.
+// slot; the CTA that finishes the last partial of a unit (an atomic ticket, no waiting)
+// merges the unit's partials by their log-sum-exp and writes out/lse.
 //
 // The kernel is HBM-bound by design: ~32 issue slots per 8 KB of KV per warp; what matters
 // is the depth of the TMA ring (192 KB in flight per SM) and that nothing stalls the
@@ -35,7 +36,9 @@ namespace {
 
 constexpr int kStages = 6;
 constexpr int kConsumerWarps = 4;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kProducerWarp = kConsumerWarps;          // warp 4
+constexpr int kCombinerWarp = kConsumerWarps + 1;      // warp 5
+constexpr int kThreads = (kConsumerWarps + 2) * 32;
 constexpr int kTileBytes = kTile * kRowBytes;             // 16 KB: one K or V tile
 constexpr int kQBytes = kGroup * kRowBytes;               // 2 KB: the 8 query rows of a group
 constexpr int kStageBytes = 2 * kTileBytes + kQBytes;     // K | V | Q
@@ -48,7 +51,16 @@ struct StageMeta {
     int32_t b, g, slot;
     int32_t n_valid;       // valid tokens in the tile (1..64); 0 = no more work
     int32_t first, last;   // first / last tile of its segment
-    int32_t pad0, pad1;
+    int32_t unit_start;    // flat tile index of the unit's first tile
+    int32_t tiles_b;       // tiles of the whole unit
+};
+
+// A finished partial segment handed from the consumer warps to the combiner warp.
+struct CombineJob {
+    int32_t b, g;
+    int32_t unit_start, tiles_b;
+    int32_t exit;          // 1 = the consumers are done; the combiner warp leaves
+    int32_t pad[3];
 };
 
 struct Smem {
@@ -59,9 +71,10 @@ struct Smem {
     static constexpr int kPrefixOff = kMlOff + kConsumerWarps * kGroup * 2 * 4;  // [kSmemBatch + 1]
     static constexpr int kLenOff = kPrefixOff + (kSmemBatch + 1) * 4;            // [kSmemBatch + 1]
     static constexpr int kMetaOff = kLenOff + (kSmemBatch + 1) * 4;
-    static constexpr int kBarOff = kMetaOff + kStages * (int)sizeof(StageMeta);  // full_k, full_v, empty, merge x2
-    static constexpr int kAbortOff = kBarOff + (3 * kStages + 2) * 8;
-    static constexpr int kTotal = kAbortOff + 16;
+    static constexpr int kBarOff = kMetaOff + kStages * (int)sizeof(StageMeta);  // full_k, full_v, empty, merge x2, job x2
+    static constexpr int kAbortOff = kBarOff + (3 * kStages + 4) * 8;            // abort flag
+    static constexpr int kJobOff = kAbortOff + 16;                               // CombineJob
+    static constexpr int kTotal = kJobOff + 32;
 };
 constexpr int kSmemBytes = Smem::kTotal + 1024;           // slack for the manual 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
@@ -106,6 +119,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             else if (now - t0 > kWaitLimitNs) return false;
         }
     }
+}
+// Records a wait that ran out: sticky flag, first failing site, CTA-wide abort.
+__device__ __forceinline__ void wait_failed(const DecodeParams& p, volatile int32_t* abort_flag, int site) {
+    *abort_flag = 1;
+    atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+    atomicCAS(p.hdr + kHdrWaitSite, 0, site);
 }
 __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int32_t row, uint32_t bar) {
     // box {64 elements, P rows, 2 halves} at coordinates {0, row, 0}
@@ -169,11 +188,12 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
     const uint32_t merge_bar0 = bar_base + 8u * (3 * kStages);
     const uint32_t merge_bar1 = merge_bar0 + 8u;
+    const uint32_t job_ready = merge_bar0 + 16u;      // consumers -> combiner: a job is posted
+    const uint32_t job_taken = merge_bar0 + 24u;      // combiner -> consumers: the job slot is free again
+    volatile CombineJob* job_s = reinterpret_cast<volatile CombineJob*>(smem + Smem::kJobOff);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int32_t W = p.hdr[kHdrTotalTiles];
-    const int32_t R = p.hdr[kHdrNumRanges];
     const int32_t P = p.page_size;
     const int64_t max_len = (int64_t)p.bt_stride * P;
     const bool cached = p.batch <= kSmemBatch;
@@ -186,10 +206,17 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         }
         mbar_init(merge_bar0, kConsumerWarps * 32);
         mbar_init(merge_bar1, kConsumerWarps * 32);
+        mbar_init(job_ready, kConsumerWarps * 32);
+        mbar_init(job_taken, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // everything above overlaps the plan kernel when launched as its programmatic dependent;
+    // the plan's outputs are read only below this wait
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int32_t W = p.hdr[kHdrTotalTiles];
+    const int32_t R = p.hdr[kHdrNumRanges];
     if (cached) {
         for (int i = tid; i <= p.batch; i += kThreads) sm_prefix[i] = p.tiles_prefix[i];
         for (int i = tid; i < p.batch; i += kThreads) {
@@ -200,21 +227,20 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     __syncthreads();
     const int32_t* prefix = cached ? sm_prefix : p.tiles_prefix;
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // =========================================================== producer warp
         uint32_t it = 0;                       // tiles issued so far
-        int32_t r = 0;
-        if (lane == 0) r = atomicAdd(p.hdr + kHdrClaim, 1);
-        r = __shfl_sync(0xffffffffu, r, 0);
+        int32_t r = blockIdx.x;                // CTA i starts on range i; further ranges are claimed
         bool ok = true;
         const int pages_per_tile_shift = 6 - p.page_shift;      // log2(64 / P)
         const uint32_t box_bytes = (uint32_t)P * kRowBytes;
         while (ok && r < R) {
-            // claim the next range now; its latency hides behind this range's copies
+            // the next range is claimed a few tiles before this one ends: late enough that no
+            // CTA sits on work another could start, early enough to hide the atomic's latency
             int32_t r_next = 0;
-            if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
-            const int32_t x0 = (int32_t)(((int64_t)W * r) / R);
-            const int32_t x1 = (int32_t)(((int64_t)W * (r + 1)) / R);
+            bool claimed = false;
+            const int32_t x0 = range_begin(W, R, r);
+            const int32_t x1 = range_begin(W, R, r + 1);
             int32_t x = x0;
             while (ok && x < x1) {
                 const Segment sg = segment_at(prefix, p.batch, r, x0, x1, x);
@@ -227,7 +253,12 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 int32_t chunk_base = (sg.tile0 << pages_per_tile_shift);
                 // this lane's entry of the current 32-page chunk of the block table
                 int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
+                const int32_t unit_start = x - sg.tile1;      // x already points past the segment
                 for (int32_t t = sg.tile0; ok && t < sg.tile1; ++t) {
+                    if (!claimed && x1 - (unit_start + t) <= p.claim_ahead) {
+                        if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
+                        claimed = true;
+                    }
                     const int32_t first_page = t << pages_per_tile_shift;
                     if (first_page >= chunk_base + 32) {
                         chunk_base = first_page;
@@ -254,6 +285,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                             StageMeta& m = meta[s];
                             m.b = sg.b; m.g = sg.g; m.slot = sg.slot; m.n_valid = n_valid;
                             m.first = (t == sg.tile0); m.last = (t == sg.tile1 - 1);
+                            m.unit_start = unit_start; m.tiles_b = sg.tiles_b;
                             const uint32_t kdst = smem_base + s * kStageBytes;
                             const uint32_t vdst = kdst + kTileBytes;
                             const bool with_q = (t == sg.tile0);
@@ -291,8 +323,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 }
             }
             if (!ok) {
-                *abort_flag = 1;
-                atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                wait_failed(p, abort_flag, 1);
                 // let the copies still in flight land before the CTA's shared memory is released
                 const uint32_t lo = it > (uint32_t)kStages ? it - kStages : 0u;
                 for (uint32_t j = lo; j < it; ++j) {
@@ -303,6 +334,74 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             }
         }
         return;
+    }
+
+    if (warp == kCombinerWarp) {
+        // =========================================================== combiner warp
+        // Takes the jobs the consumers post.  Each job is one finished partial of a unit that
+        // the plan split over several ranges: an atomic ticket on the unit's counter tells
+        // whether it was the unit's last one, and if so this warp merges the unit's partials
+        //   L = log2 sum_s 2^{lse_s},  out = sum_s 2^{lse_s - L} out_s,  lse = L ln 2
+        // with a running maximum, 4 dims per lane, all 8 heads in flight at once.
+        const float ninf_c = -INFINITY;
+        for (uint32_t jobn = 0;; ++jobn) {
+            if (!mbar_wait(job_ready, jobn & 1u, abort_flag)) {
+                if (lane == 0) wait_failed(p, abort_flag, 8);
+                return;
+            }
+            const int32_t jb = job_s->b, jg = job_s->g, ju = job_s->unit_start, jt = job_s->tiles_b;
+            const int32_t jexit = job_s->exit;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(job_taken);
+            if (jexit) return;
+            int32_t ticket = 0;
+            if (lane == 0)
+                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;"
+                             : "=r"(ticket) : "l"(p.unit_done + jb * kHkv + jg), "r"(1) : "memory");
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            __syncwarp();
+            const int32_t r_lo = range_of(W, R, ju);
+            const int32_t r_hi = range_of(W, R, ju + jt - 1);
+            const int32_t splits = r_hi - r_lo + 1;
+            if (ticket != splits - 1) continue;
+            // the unit's segment in range r is that range's first (slot 2r) unless the range
+            // began before the unit did, which can only be the case for r_lo
+            const int32_t slot_lo = 2 * r_lo + (range_begin(W, R, r_lo) < ju ? 1 : 0);
+            float mx[kGroup], z[kGroup];
+            float4 acc[kGroup];
+            #pragma unroll
+            for (int h = 0; h < kGroup; ++h) { mx[h] = ninf_c; z[h] = 0.f; acc[h] = make_float4(0.f, 0.f, 0.f, 0.f); }
+            #pragma unroll 2
+            for (int32_t i = 0; i < splits; ++i) {
+                const int64_t slot = i ? 2 * (int64_t)(r_lo + i) : slot_lo;
+                const float4* lp = reinterpret_cast<const float4*>(p.part_lse + slot * kGroup);
+                const float4 la = __ldcg(lp), lb = __ldcg(lp + 1);
+                const float l8[kGroup] = {la.x, la.y, la.z, la.w, lb.x, lb.y, lb.z, lb.w};
+                float4 v[kGroup];
+                #pragma unroll
+                for (int h = 0; h < kGroup; ++h)
+                    v[h] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (slot * kGroup + h) * kD) + lane);
+                #pragma unroll
+                for (int h = 0; h < kGroup; ++h) {
+                    const float mn = fmaxf(mx[h], l8[h]);
+                    const float a = fast_exp2(mx[h] - mn), wt = fast_exp2(l8[h] - mn);
+                    mx[h] = mn;
+                    z[h] = fmaf(z[h], a, wt);
+                    acc[h].x = fmaf(acc[h].x, a, wt * v[h].x); acc[h].y = fmaf(acc[h].y, a, wt * v[h].y);
+                    acc[h].z = fmaf(acc[h].z, a, wt * v[h].z); acc[h].w = fmaf(acc[h].w, a, wt * v[h].w);
+                }
+            }
+            #pragma unroll
+            for (int h = 0; h < kGroup; ++h) {
+                const float inv = 1.f / z[h];
+                const int64_t row = (int64_t)jb * kHq + jg * kGroup + h;
+                uint2 packed;
+                packed.x = pack_bf16(acc[h].x * inv, acc[h].y * inv);
+                packed.y = pack_bf16(acc[h].z * inv, acc[h].w * inv);
+                reinterpret_cast<uint2*>(p.out + row * kD)[lane] = packed;
+                if (lane == 0) p.lse[row] = (mx[h] + log2f(z[h])) * 0.6931471805599453f;
+            }
+        }
     }
 
     // =============================================================== consumer warps
@@ -330,18 +429,32 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     float o[8][4];
     #pragma unroll
     for (int i = 0; i < 8; ++i) { qf[i][0] = qf[i][1] = 0u; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    uint32_t merges = 0;
+    uint32_t merges = 0, jobs = 0;
 
     for (uint32_t it = 0;; ++it) {
         const int s = it % kStages;
         const uint32_t parity = (it / kStages) & 1u;
         if (!mbar_wait(full_k(s), parity, abort_flag)) {
-            *abort_flag = 1;
-            if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
-            return;
+                if (lane == 0) wait_failed(p, abort_flag, 2);
+                return;
         }
         const StageMeta mt = meta[s];
-        if (mt.n_valid == 0) return;
+        if (mt.n_valid == 0) {
+            // no more work: tell the combiner warp to leave once it has taken the last job.
+            // All consumer threads meet first, so that no exit arrival can be counted into a
+            // job phase that thread 0 (which may still be waiting to post it) has not joined.
+            mbar_arrive(merge_bar0);
+            if (!mbar_wait(merge_bar0, merges & 1u, abort_flag)) {
+                if (lane == 0) wait_failed(p, abort_flag, 9);
+                return;
+            }
+            if (tid == 0) {
+                if (mbar_wait(job_taken, (jobs & 1u) ^ 1u, abort_flag)) job_s->exit = 1;
+                else wait_failed(p, abort_flag, 7);
+            }
+            mbar_arrive(job_ready);
+            return;
+        }
         const uint32_t kbase = smem_base + s * kStageBytes;
         const uint32_t vbase = kbase + kTileBytes;
         if (mt.first) {
@@ -397,8 +510,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             const uint32_t pb1 = movmatrix_trans(pack_bf16(p10, p11));
 
             if (!mbar_wait(full_v(s), parity, abort_flag)) {
-                *abort_flag = 1;
-                if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                if (lane == 0) wait_failed(p, abort_flag, 3);
                 return;
             }
             if (valid < 16) {
@@ -450,8 +562,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             }
             mbar_arrive(merge_bar0);
             if (!mbar_wait(merge_bar0, merges & 1u, abort_flag)) {
-                *abort_flag = 1;
-                if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                if (lane == 0) wait_failed(p, abort_flag, 4);
                 return;
             }
             const int d = tid;                        // 128 consumer threads = 128 dims
@@ -481,9 +592,18 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             }
             mbar_arrive(merge_bar1);
             if (!mbar_wait(merge_bar1, merges & 1u, abort_flag)) {
-                *abort_flag = 1;
-                if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
+                if (lane == 0) wait_failed(p, abort_flag, 5);
                 return;
+            }
+            if (mt.slot >= 0 && p.fuse_combine) {
+                // hand the finished partial to the combiner warp; nobody here waits for it
+                if (tid == 0) {
+                    if (!mbar_wait(job_taken, (jobs & 1u) ^ 1u, abort_flag)) wait_failed(p, abort_flag, 6);
+                    job_s->b = mt.b; job_s->g = mt.g; job_s->unit_start = mt.unit_start;
+                    job_s->tiles_b = mt.tiles_b; job_s->exit = 0;
+                }
+                mbar_arrive(job_ready);       // releases this thread's partial stores to the combiner warp
+                ++jobs;
             }
             ++merges;
         }
@@ -544,8 +664,18 @@ cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
     if (!make_pool_map(&map_k, p.k_pages, p.num_pages, p.page_size) ||
         !make_pool_map(&map_v, p.v_pages, p.num_pages, p.page_size))
         return cudaErrorInvalidValue;
-    partial_mma_kernel<<<p.grid_ctas, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
-    return cudaGetLastError();
+    // programmatic dependent launch: the prologue (barrier set-up) may overlap the plan kernel
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.grid_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, partial_mma_kernel, p, map_k, map_v);
 }
 
 }  // namespace concur

@@ -41,12 +41,8 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
     const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
     const float ninf = -INFINITY;
 
-    for (;;) {
-        __syncthreads();
-        if (tid == 0) claim_s = atomicAdd(p.hdr + kHdrClaim, 1);
-        __syncthreads();
-        const int32_t r = claim_s;
-        if (r >= R) break;
+    // CTA i starts on range i; every further range is claimed from the shared counter
+    for (int32_t r = blockIdx.x; r < R;) {
         const int32_t x0 = p.range_start[r], x1 = p.range_start[r + 1];
         int32_t x = x0;
         while (x < x1) {
@@ -187,6 +183,10 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
                 }
             }
         }
+        __syncthreads();
+        if (tid == 0) claim_s = atomicAdd(p.hdr + kHdrClaim, 1);
+        __syncthreads();
+        r = claim_s;
     }
 }
 

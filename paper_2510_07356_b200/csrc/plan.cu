@@ -18,6 +18,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
     __shared__ int32_t ranges_s;
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
+    // lets a dependent launch (programmatic stream serialisation) start its prologue now; it
+    // still waits for this grid to finish before it reads the plan
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) { carry_s = 0; p.tiles_prefix[0] = 0; }
     __syncthreads();
 
@@ -31,6 +34,17 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
             if (len < 0) { len = 0; flags |= kFlagBadLen; }
             if (len > max_len) { len = max_len; flags |= kFlagBadLen; }
             tiles = (int32_t)((len + kTile - 1) / kTile);
+        }
+        // sequences without cached tokens get their result here (out = 0, lse = -inf): the
+        // warp that found one writes it
+        unsigned empties = __ballot_sync(0xffffffffu, b < p.batch && tiles == 0);
+        while (empties) {
+            const int e = base + warp * 32 + (__ffs(empties) - 1);
+            empties &= empties - 1;
+            uint4* o = reinterpret_cast<uint4*>(p.out + (int64_t)e * kHq * kD);
+            for (int i = lane; i < kHq * kD / 8; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+            p.lse[(int64_t)e * kHq + lane] = -INFINITY;
+            p.lse[(int64_t)e * kHq + 32 + lane] = -INFINITY;
         }
         // inclusive scan over the block
         int32_t v = tiles;
@@ -58,6 +72,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
         __syncthreads();
     }
     if (flags) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), flags);
+    for (int i = tid; i < p.batch * kHkv; i += kPlanThreads) p.unit_done[i] = 0;
 
     if (tid == 0) {
         const int32_t W = kHkv * carry_s;
@@ -76,7 +91,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
         if (R < 1 && W > 0) R = 1;
         p.hdr[kHdrTotalTiles] = W;
         p.hdr[kHdrNumRanges] = R;
-        p.hdr[kHdrClaim] = 0;
+        p.hdr[kHdrClaim] = p.grid_ctas;       // CTA i starts on range i; further ranges are claimed from here
         ranges_s = R;
     }
     __syncthreads();

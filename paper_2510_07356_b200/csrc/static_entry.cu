@@ -28,7 +28,8 @@ constexpr size_t round256(size_t x) { return (x + 255) / 256 * 256; }
 constexpr size_t kOffHdr = 0;
 constexpr size_t kOffPrefix = kOffHdr + round256(kHdrWords * sizeof(int32_t));
 constexpr size_t kOffRangeStart = kOffPrefix + round256((kStaticMaxBatch + 1) * sizeof(int32_t));
-constexpr size_t kOffPartLse = kOffRangeStart + round256((kStaticMaxRanges + 1) * sizeof(int32_t));
+constexpr size_t kOffUnitDone = kOffRangeStart + round256((kStaticMaxRanges + 1) * sizeof(int32_t));
+constexpr size_t kOffPartLse = kOffUnitDone + round256((size_t)kStaticMaxBatch * kHkv * sizeof(int32_t));
 constexpr size_t kOffPartO = kOffPartLse + round256((size_t)2 * kStaticMaxRanges * kGroup * sizeof(float));
 constexpr size_t kStaticBytes = kOffPartO + round256((size_t)2 * kStaticMaxRanges * kGroup * kD * sizeof(float));
 
@@ -105,21 +106,23 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.page_shift = page_size == 16 ? 4 : (page_size == 32 ? 5 : 6);
     p.grid_ctas = s->sm_count;
     p.forced_ranges = 0;
-    p.ranges_per_cta = 16;
+    p.ranges_per_cta = 1;
     p.min_range_tiles = 2;
     p.max_ranges = kStaticMaxRanges;
-    // the plan kernel rewrites the tile count, the range count and the claim counter at the
-    // start of every call, and every partial slot is written before the combine kernel reads
-    // it, so nothing of the previous call's contents has to be cleared here
+    p.fuse_combine = 1;
+    p.claim_ahead = 1 << 20;
+    // the plan kernel rewrites the tile count, the range count, the claim counter and the
+    // per-unit counters at the start of every call, and every partial slot is written before
+    // it is read, so nothing of the previous call's contents has to be cleared here
     p.hdr = reinterpret_cast<int32_t*>(s->scratch + kOffHdr);
     p.tiles_prefix = reinterpret_cast<int32_t*>(s->scratch + kOffPrefix);
     p.range_start = reinterpret_cast<int32_t*>(s->scratch + kOffRangeStart);
+    p.unit_done = reinterpret_cast<int32_t*>(s->scratch + kOffUnitDone);
     p.part_lse = reinterpret_cast<float*>(s->scratch + kOffPartLse);
     p.part_o = reinterpret_cast<float*>(s->scratch + kOffPartO);
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (launch_plan(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if (launch_partial_mma(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
-    if (launch_combine(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     return CONCUR_OK;
 }
