@@ -30,6 +30,10 @@ UNIT = "GB/s"
 DEFAULT_WORKLOAD = "cfg3_b64_ctx16384_p64"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one partial_mma_kernel launch divided by its KV tokens, from
+# the ncu capture summarised in profiles/partial_mma_cfg3q_b16_ctx16384.md (page size 64, fused combine, one
+# range per CTA).  Set to None whenever that kernel changes until the counters are taken again.
+MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074916e9 + 5.105664e6) / 262144
 
 
 def parse_args():
@@ -376,6 +380,9 @@ def main():
     peak, peak_kind = measured_peak()
     value = world * nbytes / (ms_per_step * 1e-3) / 1e9
     achieved = nbytes / (part_ms_avg * 1e-3) / 1e9
+    traffic = None
+    if args.kernel == 0 and spec.page_size == 64 and MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN:
+        traffic = MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN * w.kv_tokens     # scaled from the quarter-size capture
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -389,7 +396,7 @@ def main():
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "partial", "ms": part_ms_avg,
+                     "peak_kind": f"of {peak_kind}", "traffic": traffic, "kernel": "partial", "ms": part_ms_avg,
                      "ms_min": min(part_ms)},
         "step_ms_min": min(step_ms),
         "e2e": e2e, "gpu_launches": (2 if args.kernel == 0 else 3) * K, "clocks": clocks, "device_flags": flags,
