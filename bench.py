@@ -179,6 +179,25 @@ def cpu_baseline(w, target_seconds):
                       f"{dt:.1f} s wall", "kv_tokens_per_s": tok / dt}
 
 
+def rank_spec(spec, rank: int, world: int):
+    """Replicas: every rank decodes its own batch of the same shape, drawn from its own seed."""
+    if world <= 1:
+        return spec
+    from dataclasses import replace
+    return replace(spec, seed=spec.seed + 100 * rank)
+
+
+def over_ranks(values, op, device):
+    """Element-wise MAX or SUM of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return t.tolist()
+
+
 def run_reference(args):
     """The oracle timed on the host cores; rank 0 only."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -249,10 +268,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # every rank decodes its own batch of the same shape (replicas, no data-path collective)
-    spec = synth.SPECS[args.workload]
-    if world > 1:
-        from dataclasses import replace
-        spec = replace(spec, seed=spec.seed + 100 * rank)
+    spec = rank_spec(synth.SPECS[args.workload], rank, world)
     w = synth.make_workload(spec, dev)
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
     attn.set_option(P.CONCUR_OPT_KERNEL, args.kernel)
@@ -333,10 +349,8 @@ def main():
     attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, 0)
     part_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
     part_ms_avg = sum(part_ms) / K
-    if world > 1:
-        t = torch.tensor([ms_per_step, part_ms_avg], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, part_ms_avg = t.tolist()
+    ms_per_step, part_ms_avg = over_ranks([ms_per_step, part_ms_avg], "max", dev)
+    job_bytes, job_tokens = over_ranks([nbytes, w.kv_tokens], "sum", dev)     # units all ranks processed
     flags = attn.status()
     R, W, _ = attn.last_plan()
 
@@ -362,11 +376,8 @@ def main():
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = t.item()
-        e2e = {"value": world * nbytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e_ms = over_ranks([e2e_ms], "max", dev)[0]
+        e2e = {"value": job_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                "entry": "concur_decode_attn_host"}
         assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), "host path differs from device path"
@@ -378,7 +389,7 @@ def main():
         return
 
     peak, peak_kind = measured_peak()
-    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
+    value = job_bytes / (ms_per_step * 1e-3) / 1e9
     achieved = nbytes / (part_ms_avg * 1e-3) / 1e9
     traffic = None
     if args.kernel == 0 and spec.page_size == 64 and MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN:
@@ -392,7 +403,7 @@ def main():
                    "l2": "flushed between steps" if flush_needed else "inputs larger than L2",
                    "kernel": "mma" if args.kernel == 0 else "scalar", "ranges": R, "tiles": W,
                    "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
-        "kv_tokens_per_s": world * w.kv_tokens / (ms_per_step * 1e-3),
+        "kv_tokens_per_s": job_tokens / (ms_per_step * 1e-3),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -216,3 +216,22 @@ def test_subset_selection_matches_full():
     o2, l2 = oracle.decode_attn(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens, sub.scale)
     assert np.array_equal(o2[0], full[0][2]) and np.array_equal(o2[1], full[0][0])
     assert np.array_equal(l2[1], full[1][0])
+
+
+def test_frozen_tiny_case_has_not_drifted():
+    # regression fixture written by tests/golden/make_golden.py from the oracle alone
+    import importlib.util
+    import json
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "golden", "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    with open(os.path.join(here, "golden", "tiny_decode_oracle.json")) as f:
+        gold = json.load(f)
+    w, out, lse = mod.compute()
+    assert w.q.view(-1)[:8].view(dtype=torch.int16).tolist() == gold["q_first_bits"], "input generator drifted"
+    np.testing.assert_allclose(lse, np.array([[float(x) for x in r] for r in gold["lse"]]), rtol=1e-13)
+    got = np.array([[out[b, h, :4] for h in range(0, 64, 8)] for b in range(4)])
+    want = np.array([[[float(x) for x in hrow] for hrow in brow] for brow in gold["out_first4"]])
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
