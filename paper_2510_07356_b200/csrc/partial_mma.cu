@@ -251,8 +251,10 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 const int32_t* table = p.block_table + (int64_t)sg.b * p.bt_stride;
                 const int32_t page_end = (min(sg.tile1 * kTile, n) + P - 1) >> p.page_shift;   // pages used by the segment
                 int32_t chunk_base = (sg.tile0 << pages_per_tile_shift);
-                // this lane's entry of the current 32-page chunk of the block table
+                // this lane's entry of the current 32-page chunk of the block table, and of the
+                // chunk after it (fetched one chunk early so that its latency never stalls the ring)
                 int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
+                int32_t pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                 const int32_t unit_start = x - sg.tile1;      // x already points past the segment
                 for (int32_t t = sg.tile0; ok && t < sg.tile1; ++t) {
                     if (!claimed && x1 - (unit_start + t) <= p.claim_ahead) {
@@ -261,8 +263,9 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                     }
                     const int32_t first_page = t << pages_per_tile_shift;
                     if (first_page >= chunk_base + 32) {
-                        chunk_base = first_page;
-                        pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
+                        chunk_base += 32;
+                        pg = pg_next;
+                        pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                     }
                     const int32_t n_valid = min(kTile, n - t * kTile);
                     const int32_t npages = (n_valid + P - 1) >> p.page_shift;

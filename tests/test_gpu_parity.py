@@ -246,3 +246,43 @@ def test_host_entry_point_matches_device_entry_point(P):
     assert torch.equal(out_h.view(torch.int16), out_d.cpu().view(torch.int16))
     assert torch.equal(lse_h, lse_d.cpu())
     attn.close()
+
+
+@pytest.mark.parametrize("kernel", list(KERNELS))
+def test_many_short_sequences(P, kernel):
+    # more sequences than the partial kernel caches plan rows for (it then reads them from
+    # global memory), a third of them empty or shorter than one page
+    rng = np.random.default_rng(2024)
+    lens = rng.integers(0, 400, size=700)
+    lens[rng.integers(0, 700, size=60)] = 0
+    lens[rng.integers(0, 700, size=60)] = rng.integers(1, 16, size=60)
+    spec = synth.tiny_spec("many", [int(x) for x in lens], 16, 88)
+    w = synth.make_workload(spec, "cuda:0")
+    out, lse, attn = run(P, w, KERNELS[kernel])
+    assert attn.status() == 0
+    ref_out, ref_lse = oracle_sequences(to_host(w))
+    assert_parity(out, lse, ref_out, ref_lse, f"{kernel} 700 sequences")
+    attn.close()
+
+
+def test_repeated_calls_on_one_handle_are_identical(P):
+    # the workspace is reused call after call: counters and partial slots of an earlier,
+    # larger call must not leak into a later one
+    big = synth.make_workload(synth.tiny_spec("rep_big", (9000, 300, 4097), 64, 41), "cuda:0")
+    small = synth.make_workload(synth.tiny_spec("rep_small", (130, 64), 64, 42), "cuda:0")
+    attn = P.DecodeAttention(64, 3, max(big.block_table.shape[1], small.block_table.shape[1]), 0)
+    first = None
+    for _ in range(3):
+        ob, lb = attn(big.q, big.k_pages, big.v_pages, big.block_table, big.seq_lens, big.scale)
+        os_, ls = attn(small.q, small.k_pages, small.v_pages, small.block_table, small.seq_lens, small.scale)
+        torch.cuda.synchronize()
+        if first is None:
+            first = (ob.clone(), lb.clone(), os_.clone(), ls.clone())
+        else:
+            for a, b in zip(first, (ob, lb, os_, ls)):
+                assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                                   b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+    ref_out, ref_lse = oracle_sequences(to_host(small))
+    assert_parity(first[2], first[3], ref_out, ref_lse, "small after big")
+    assert attn.status() == 0
+    attn.close()
