@@ -135,6 +135,29 @@ int concur_decode_attn(concur_attn_t* handle,
                        void* cuda_stream);
 
 /*
+ * The write path of the paged cache, run once per decode step before the attention call:
+ * for every sequence b, the new token's rows k_new[b][g][:], v_new[b][g][:] (g = 0..Hkv-1)
+ * are stored at position pos = seq_lens[b], i.e. slot pos % P of page
+ * block_table[b][pos / P], and seq_lens[b] becomes pos + 1.  (The generation loop whose
+ * attention step this library implements -- Sec. 3.3 / 4.1 of the paper -- appends one
+ * token per sequence per step; the paper does not describe the cache.)
+ *
+ *   k_new, v_new   device, bf16 [batch][Hkv][D], 16-byte aligned
+ *   k_pages, v_pages, block_table   as for concur_decode_attn (the pools are written)
+ *   seq_lens       device, int32 [batch], read and advanced
+ *
+ * Asynchronous on `cuda_stream`.  A sequence whose position is outside [0, stride*P) or
+ * whose page id is outside [0, num_pages) is left untouched (nothing written, length not
+ * advanced) and CONCUR_FLAG_BAD_SEQ_LEN / CONCUR_FLAG_BAD_PAGE_ID is recorded.  The page
+ * must already be allocated in the block table: page allocation is the caller's.
+ * Errors as for concur_decode_attn.
+ */
+int concur_kv_append(concur_attn_t* handle, const void* k_new, const void* v_new,
+                     void* k_pages, void* v_pages, const int32_t* block_table, int32_t* seq_lens,
+                     int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                     void* cuda_stream);
+
+/*
  * The same step for callers whose tensors live in HOST memory (pinned memory gives
  * asynchronous copies).  Every pointer is a host pointer with the layouts above; the
  * library copies the inputs into device staging buffers that it owns (allocated on first

@@ -36,7 +36,7 @@ EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
-    "concur_decode_attn_static",
+    "concur_decode_attn_static", "concur_kv_append",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -71,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_decode_attn_host.argtypes = decode_args
     lib.concur_decode_attn_static.restype = ctypes.c_int
     lib.concur_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
+    lib.concur_kv_append.restype = ctypes.c_int
+    lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
     lib.concur_attn_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.concur_attn_set_option.restype = ctypes.c_int
@@ -164,6 +166,17 @@ def concur_decode_attn_static(q, k_pages, v_pages, block_table, seq_lens, scale,
                                        batch, num_pages, block_table_stride, page_size, stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_decode_attn_static")
+    return rc
+
+
+def concur_kv_append(handle, k_new, v_new, k_pages, v_pages, block_table, seq_lens, batch, num_pages,
+                     block_table_stride, stream=0, check=True) -> int:
+    """Stores each sequence's new K/V rows at position seq_lens[b] and advances seq_lens (device tensors)."""
+    rc = lib.concur_kv_append(handle, _addr(k_new), _addr(v_new), _addr(k_pages), _addr(v_pages),
+                              _addr(block_table), _addr(seq_lens), batch, num_pages, block_table_stride,
+                              stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_kv_append")
     return rc
 
 

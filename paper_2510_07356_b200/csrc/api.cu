@@ -206,6 +206,29 @@ int concur_decode_attn(concur_attn_t* h, const void* q, const void* k_pages, con
     return enqueue(h, p, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
+                     const int32_t* block_table, int32_t* seq_lens, int32_t batch, int32_t num_pages,
+                     int32_t block_table_stride, void* cuda_stream) {
+    if (!h) return CONCUR_ERR_INVALID_ARG;
+    if (batch < 0 || num_pages < 1 || block_table_stride < 1) return CONCUR_ERR_INVALID_ARG;
+    if (batch > h->cfg.max_batch || block_table_stride > h->cfg.max_pages_per_seq) return CONCUR_ERR_TOO_LARGE;
+    if ((int64_t)num_pages * kHkv * h->cfg.page_size >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
+    if (batch == 0) return CONCUR_OK;
+    if (!k_new || !v_new || !k_pages || !v_pages || !block_table || !seq_lens) return CONCUR_ERR_INVALID_ARG;
+    if (!aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(k_pages, 16) || !aligned(v_pages, 16) ||
+        !aligned(block_table, 4) || !aligned(seq_lens, 4))
+        return CONCUR_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok()) return CONCUR_ERR_CUDA;
+    const int32_t P = h->cfg.page_size;
+    const int32_t shift = P == 16 ? 4 : (P == 32 ? 5 : 6);
+    if (launch_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
+                      reinterpret_cast<int32_t*>(h->ws + h->lay.hdr), batch, num_pages, block_table_stride, P,
+                      shift, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return CONCUR_ERR_CUDA;
+    return CONCUR_OK;
+}
+
 static int ensure(Staging& s, size_t bytes) {
     if (bytes <= s.cap) return CONCUR_OK;
     if (s.ptr) cudaFree(s.ptr);

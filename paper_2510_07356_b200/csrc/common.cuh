@@ -127,5 +127,9 @@ cudaError_t launch_partial_scalar(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream);
 int partial_scalar_ctas_per_sm();
+cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
+                          const int32_t* block_table, int32_t* seq_lens, int32_t* hdr, int32_t batch,
+                          int32_t num_pages, int32_t bt_stride, int32_t page_size, int32_t page_shift,
+                          cudaStream_t stream);
 
 }  // namespace concur
