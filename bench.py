@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--ranges-per-cta", type=int, default=0)
     ap.add_argument("--min-range-tiles", type=int, default=0)
     ap.add_argument("--num-ranges", type=int, default=0)
+    ap.add_argument("--loop-steps", type=int, default=16, help="append+attention steps replayed from a CUDA graph")
     ap.add_argument("--fuse-combine", type=int, default=-1)
     ap.add_argument("--claim-ahead", type=int, default=-1)
     return ap.parse_args()
@@ -269,7 +270,7 @@ def main():
 
     # every rank decodes its own batch of the same shape (replicas, no data-path collective)
     spec = rank_spec(synth.SPECS[args.workload], rank, world)
-    w = synth.make_workload(spec, dev)
+    w = synth.make_workload(spec, dev, spare_tokens=args.loop_steps)
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
     attn.set_option(P.CONCUR_OPT_KERNEL, args.kernel)
     attn.set_option(P.CONCUR_OPT_RANGES_PER_CTA, args.ranges_per_cta)
@@ -383,6 +384,34 @@ def main():
         assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), "host path differs from device path"
         del hq, hk, hv
 
+    # ---- decode loop: KV append + attention per step, replayed from one CUDA graph
+    loop = None
+    if args.loop_steps > 0:
+        g = torch.Generator(device=dev); g.manual_seed(spec.seed + 17)
+        kn = torch.randn((spec.batch, spec.num_kv_heads, spec.head_dim), generator=g, device=dev).to(torch.bfloat16)
+        vn = torch.randn((spec.batch, spec.num_kv_heads, spec.head_dim), generator=g, device=dev).to(torch.bfloat16)
+        lens_loop = w.seq_lens.clone()
+
+        def loop_step():
+            s_ = torch.cuda.current_stream(dev).cuda_stream
+            P.concur_kv_append(attn.handle, kn, vn, w.k_pages, w.v_pages, w.block_table, lens_loop, spec.batch,
+                               w.num_pages, w.block_table.shape[1], s_)
+            attn(w.q, w.k_pages, w.v_pages, w.block_table, lens_loop, w.scale, out=out, lse=lse)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            loop_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.loop_steps):
+            graph.replay()
+        e1.record(stream)
+        barrier()
+        loop_ms = over_ranks([e0.elapsed_time(e1) / args.loop_steps], "max", dev)[0]
+        assert int(lens_loop[0]) == int(w.lens_host[0]) + args.loop_steps
+        loop = {"steps": args.loop_steps, "ms_per_step": loop_ms, "launches_per_step": 3,
+                "what": "concur_kv_append + concur_decode_attn replayed from a CUDA graph, lengths +1 per step"}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -410,7 +439,7 @@ def main():
                      "peak_kind": f"of {peak_kind}", "traffic": traffic, "kernel": "partial", "ms": part_ms_avg,
                      "ms_min": min(part_ms)},
         "step_ms_min": min(step_ms),
-        "e2e": e2e, "gpu_launches": (2 if args.kernel == 0 else 3) * K, "clocks": clocks, "device_flags": flags,
+        "decode_loop": loop, "e2e": e2e, "gpu_launches": (2 if args.kernel == 0 else 3) * K, "clocks": clocks, "device_flags": flags,
     }
     if not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)

@@ -90,7 +90,7 @@ class Workload:
         s = self.spec
         per_token = 2 * s.num_kv_heads * s.head_dim * 2
         per_seq = 2 * s.num_q_heads * s.head_dim * 2 + s.num_q_heads * 4
-        pages = int(np.sum((self.lens_host + s.page_size - 1) // s.page_size))
+        pages = int(np.sum((self.lens_host.astype(np.int64) + s.page_size - 1) // s.page_size))
         return self.kv_tokens * per_token + s.batch * (per_seq + 4) + pages * 4
 
 
@@ -123,10 +123,11 @@ def make_lengths(spec: Spec) -> np.ndarray:
     return lens.astype(np.int32)
 
 
-def make_block_table(spec: Spec, lens: np.ndarray, stride: int | None = None):
-    """Returns (table [B][stride] int32 with -1 tails, num_pages)."""
+def make_block_table(spec: Spec, lens: np.ndarray, stride: int | None = None, spare_tokens: int = 0):
+    """Returns (table [B][stride] int32 with -1 tails, num_pages).  `spare_tokens` allocates room
+    for that many more tokens per sequence (pages a decode loop will append into)."""
     P = spec.page_size
-    pages_per_seq = (lens.astype(np.int64) + P - 1) // P
+    pages_per_seq = (lens.astype(np.int64) + spare_tokens + P - 1) // P
     total = int(pages_per_seq.sum())
     perm = np.arange(total, dtype=np.int64)
     if spec.permute_pages:
@@ -154,12 +155,13 @@ def _normal_bf16(shape, std, gen, device, chunk_elems=1 << 28):
     return out
 
 
-def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = None) -> Workload:
+def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = None,
+                  spare_tokens: int = 0) -> Workload:
     if isinstance(spec, str):
         spec = SPECS[spec]
     device = torch.device(device)
     lens = make_lengths(spec)
-    table, num_pages = make_block_table(spec, lens, table_stride)
+    table, num_pages = make_block_table(spec, lens, table_stride, spare_tokens)
     Hq, Hkv, D, P = spec.num_q_heads, spec.num_kv_heads, spec.head_dim, spec.page_size
 
     def gen(stream):
@@ -184,7 +186,7 @@ def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = Non
     else:
         k = _normal_bf16((num_pages, Hkv, P, D), 1.0, gen(4), device)
 
-    # poison the slots past each sequence's end in its last page
+    # poison the slots past each sequence's end: the rest of its last page and any spare pages
     nan = torch.tensor(float("nan"), dtype=torch.bfloat16, device=device)
     for b, n in enumerate(lens):
         n = int(n)
@@ -192,6 +194,10 @@ def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = Non
             page = int(table[b, (n - 1) // P])
             k[page, :, n % P:, :] = nan
             v[page, :, n % P:, :] = nan
+        if spare_tokens:
+            spare = torch.from_numpy(table[b, (n + P - 1) // P:(n + spare_tokens + P - 1) // P].astype(np.int64)).to(device)
+            k[spare] = nan
+            v[spare] = nan
 
     return Workload(
         spec=spec, q=q, k_pages=k, v_pages=v,
