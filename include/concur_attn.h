@@ -135,6 +135,40 @@ int concur_decode_attn(concur_attn_t* handle,
                        void* cuda_stream);
 
 /*
+ * The same step when sequences share a cached prefix (cascade decode).  In the paper's
+ * workload every task is sampled 5 times for synthesis and 10 times for evaluation from one
+ * fixed prompt (Sec. 3.3, Sec. 4.1, App. C), so the samples of a task have their whole
+ * prompt in common; with a paged cache they can point at the same physical pages.
+ *
+ *   group_start   device, int32 [num_groups + 1]: group i is sequences group_start[i] ..
+ *                 group_start[i+1]-1 (consecutive); group_start[0] = 0, last entry = batch
+ *   prefix_lens   device, int32 [num_groups]: the caller's promise that the first
+ *                 prefix_lens[i] tokens of all sequences of group i are the same cached
+ *                 tokens, i.e. their block-table rows agree on the pages that hold them
+ *
+ * The result is defined exactly as for concur_decode_attn on the same tables (sharing
+ * changes how often the shared tiles are read, never what is computed): the shared tiles
+ * are streamed once per group and KV head and multiplied with the query rows of up to 10
+ * sharing sequences on the tensor cores; every sequence's remaining tokens are handled as
+ * in the plain step; the partial results are merged by log-sum-exp.  Only whole 64-token
+ * tiles are shared (the rest of the prefix is read per sequence), a group's sequences
+ * beyond the tenth read everything themselves, and a prefix longer than the group's
+ * shortest sequence is cut to it and recorded as CONCUR_FLAG_BAD_SEQ_LEN.  If the promise
+ * is broken the shared part is read through the group's first sequence's table.
+ *
+ * Needs max_batch <= 4096 (CONCUR_ERR_UNSUPPORTED otherwise).  The first cascade call on a
+ * handle allocates the cascade workspace (cudaMalloc; CONCUR_ERR_OOM); make it outside any
+ * stream capture.  Other arguments, asynchrony and errors as for concur_decode_attn.
+ */
+int concur_decode_attn_cascade(concur_attn_t* handle,
+                               const void* q, const void* k_pages, const void* v_pages,
+                               const int32_t* block_table, const int32_t* seq_lens,
+                               const int32_t* group_start, const int32_t* prefix_lens,
+                               float scale, void* out, float* lse,
+                               int32_t batch, int32_t num_groups, int32_t num_pages,
+                               int32_t block_table_stride, void* cuda_stream);
+
+/*
  * The write path of the paged cache, run once per decode step before the attention call:
  * for every sequence b, the new token's rows k_new[b][g][:], v_new[b][g][:] (g = 0..Hkv-1)
  * are stored at position pos = seq_lens[b], i.e. slot pos % P of page

@@ -36,7 +36,7 @@ EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
-    "concur_decode_attn_static", "concur_kv_append",
+    "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -71,6 +71,9 @@ def _load() -> ctypes.CDLL:
     lib.concur_decode_attn_host.argtypes = decode_args
     lib.concur_decode_attn_static.restype = ctypes.c_int
     lib.concur_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
+    lib.concur_decode_attn_cascade.restype = ctypes.c_int
+    lib.concur_decode_attn_cascade.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp,
+                                               i32, i32, i32, i32, vp]
     lib.concur_kv_append.restype = ctypes.c_int
     lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
@@ -166,6 +169,19 @@ def concur_decode_attn_static(q, k_pages, v_pages, block_table, seq_lens, scale,
                                        batch, num_pages, block_table_stride, page_size, stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_decode_attn_static")
+    return rc
+
+
+def concur_decode_attn_cascade(handle, q, k_pages, v_pages, block_table, seq_lens, group_start, prefix_lens,
+                               scale, out, lse, batch, num_groups, num_pages, block_table_stride,
+                               stream=0, check=True) -> int:
+    """Decode attention for groups of sequences that share a cached prefix (device tensors)."""
+    rc = lib.concur_decode_attn_cascade(handle, _addr(q), _addr(k_pages), _addr(v_pages), _addr(block_table),
+                                        _addr(seq_lens), _addr(group_start), _addr(prefix_lens),
+                                        ctypes.c_float(scale), _addr(out), _addr(lse), batch, num_groups,
+                                        num_pages, block_table_stride, stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_decode_attn_cascade")
     return rc
 
 

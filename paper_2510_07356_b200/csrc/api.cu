@@ -85,6 +85,7 @@ struct concur_attn {
     int32_t claim_ahead = 1 << 20;
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;
     Staging st_q, st_k, st_v, st_bt, st_len, st_out, st_lse;
+    Staging cascade_ws;          // allocated on the first cascade call
 };
 
 extern "C" {
@@ -160,6 +161,8 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.unit_done = reinterpret_cast<int32_t*>(h->ws + h->lay.unit_done);
     p.part_lse = reinterpret_cast<float*>(h->ws + h->lay.part_lse);
     p.part_o = reinterpret_cast<float*>(h->ws + h->lay.part_o);
+    p.tok_offset = nullptr;
+    p.all_partial = 0;
     return CONCUR_OK;
 }
 
@@ -226,6 +229,83 @@ int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, voi
                       reinterpret_cast<int32_t*>(h->ws + h->lay.hdr), batch, num_pages, block_table_stride, P,
                       shift, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return CONCUR_ERR_CUDA;
+    return CONCUR_OK;
+}
+
+static int ensure(Staging& s, size_t bytes);
+
+namespace {
+constexpr int32_t kCascadeMaxBatch = 4096;
+struct CascadeLayout {
+    size_t chdr, tok_offset, seq_group, ptiles, rowbase, pre_lse, pre_o, part_lse, part_o, total;
+    int32_t max_rows, max_slots;
+};
+CascadeLayout cascade_layout(int32_t max_batch, int sm_count) {
+    CascadeLayout w;
+    w.max_rows = kHkv * max_batch + kMaxShare * sm_count;     // whole units + one extra split per range
+    w.max_slots = kMaxRanges + kHkv * max_batch;              // suffix partial slots r + u
+    size_t at = 0;
+    w.chdr = at;        at += align_up(kHdrWords * sizeof(int32_t));
+    w.tok_offset = at;  at += align_up((size_t)max_batch * sizeof(int32_t));
+    w.seq_group = at;   at += align_up((size_t)max_batch * sizeof(int32_t));
+    w.ptiles = at;      at += align_up(((size_t)max_batch + 1) * sizeof(int32_t));
+    w.rowbase = at;     at += align_up(((size_t)max_batch * kHkv + 1) * sizeof(int32_t));
+    w.pre_lse = at;     at += align_up((size_t)w.max_rows * kGroup * sizeof(float));
+    w.pre_o = at;       at += align_up((size_t)w.max_rows * kGroup * kD * sizeof(float));
+    w.part_lse = at;    at += align_up((size_t)w.max_slots * kGroup * sizeof(float));
+    w.part_o = at;      at += align_up((size_t)w.max_slots * kGroup * kD * sizeof(float));
+    w.total = at;
+    return w;
+}
+}  // namespace
+
+int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pages, const void* v_pages,
+                               const int32_t* block_table, const int32_t* seq_lens,
+                               const int32_t* group_start, const int32_t* prefix_lens, float scale, void* out,
+                               float* lse, int32_t batch, int32_t num_groups, int32_t num_pages,
+                               int32_t block_table_stride, void* cuda_stream) {
+    int rc = check_call(h, q, k_pages, v_pages, block_table, seq_lens, out, lse, batch, num_pages,
+                        block_table_stride, 16);
+    if (rc != CONCUR_OK || batch == 0) return rc;
+    if (num_groups < 1 || num_groups > batch || !group_start || !prefix_lens || !aligned(group_start, 4) ||
+        !aligned(prefix_lens, 4))
+        return CONCUR_ERR_INVALID_ARG;
+    if (h->cfg.max_batch > kCascadeMaxBatch) return CONCUR_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok()) return CONCUR_ERR_CUDA;
+    const CascadeLayout lay = cascade_layout(h->cfg.max_batch, h->sm_count);
+    if ((rc = ensure(h->cascade_ws, lay.total)) != CONCUR_OK) return rc;
+    char* cw = static_cast<char*>(h->cascade_ws.ptr);
+
+    DecodeParams p;
+    fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
+                block_table_stride);
+    CascadeParams c;
+    c.group_start = group_start;
+    c.prefix_lens = prefix_lens;
+    c.num_groups = num_groups;
+    c.max_rows = lay.max_rows;
+    c.grid_ctas = h->sm_count;
+    c.chdr = reinterpret_cast<int32_t*>(cw + lay.chdr);
+    c.tok_offset = reinterpret_cast<int32_t*>(cw + lay.tok_offset);
+    c.seq_group = reinterpret_cast<int32_t*>(cw + lay.seq_group);
+    c.ptiles_prefix = reinterpret_cast<int32_t*>(cw + lay.ptiles);
+    c.unit_rowbase = reinterpret_cast<int32_t*>(cw + lay.rowbase);
+    c.pre_lse = reinterpret_cast<float*>(cw + lay.pre_lse);
+    c.pre_o = reinterpret_cast<float*>(cw + lay.pre_o);
+    // the suffix pass writes one partial per segment into the cascade's own slots
+    p.part_lse = reinterpret_cast<float*>(cw + lay.part_lse);
+    p.part_o = reinterpret_cast<float*>(cw + lay.part_o);
+    p.tok_offset = c.tok_offset;
+    p.all_partial = 1;
+    p.fuse_combine = 0;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (launch_plan_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    if (launch_prefix_mma(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream);
+    if (e != cudaSuccess) return CONCUR_ERR_CUDA;
+    if (launch_combine_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     return CONCUR_OK;
 }
 
@@ -352,7 +432,7 @@ int concur_attn_last_plan(concur_attn_t* h, void* cuda_stream, int32_t* num_rang
 int concur_attn_destroy(concur_attn_t* h) {
     if (!h) return CONCUR_OK;
     DeviceGuard guard(h->cfg.device);
-    Staging* all[] = {&h->st_q, &h->st_k, &h->st_v, &h->st_bt, &h->st_len, &h->st_out, &h->st_lse};
+    Staging* all[] = {&h->st_q, &h->st_k, &h->st_v, &h->st_bt, &h->st_len, &h->st_out, &h->st_lse, &h->cascade_ws};
     for (Staging* s : all) if (s->ptr) cudaFree(s->ptr);
     if (h->owns_ws && h->ws) cudaFree(h->ws);
     delete h;

@@ -52,3 +52,71 @@ cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream) {
 }
 
 }  // namespace concur
+
+// ---------------------------------------------------------------------------------------
+// Cascade combine: merges, for every (sequence, KV head) unit, the partials of its suffix
+// pass (slot r + u for every range r that covers the unit) with the partials of its group's
+// prefix pass (one row per split of the prefix unit and sharing sibling).  One pass with a
+// running maximum; all 8 heads of the group are in flight at once.
+namespace concur {
+
+__global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(DecodeParams p, CascadeParams c) {
+    const int b = blockIdx.x / kHkv, g = blockIdx.x % kHkv;
+    const int d = threadIdx.x;
+    float mx[kGroup], z[kGroup], acc[kGroup];
+    #pragma unroll
+    for (int h = 0; h < kGroup; ++h) { mx[h] = -INFINITY; z[h] = 0.f; acc[h] = 0.f; }
+    auto add = [&](const float* lse_row, const float* o_row) {
+        float l8[kGroup], v[kGroup];
+        #pragma unroll
+        for (int h = 0; h < kGroup; ++h) { l8[h] = __ldcg(lse_row + h); v[h] = __ldcg(o_row + h * kD + d); }
+        #pragma unroll
+        for (int h = 0; h < kGroup; ++h) {
+            const float mn = fmaxf(mx[h], l8[h]);
+            const float a = exp2f(mx[h] - mn), w = exp2f(l8[h] - mn);
+            mx[h] = mn;
+            z[h] = fmaf(z[h], a, w);
+            acc[h] = fmaf(acc[h], a, w * v[h]);
+        }
+    };
+    // suffix pass
+    const int32_t tiles_b = p.tiles_prefix[b + 1] - p.tiles_prefix[b];
+    if (tiles_b > 0) {
+        const int32_t W = p.hdr[kHdrTotalTiles], R = p.hdr[kHdrNumRanges];
+        const int32_t unit_start = kHkv * p.tiles_prefix[b] + g * tiles_b;
+        const int32_t r_lo = range_of(W, R, unit_start), r_hi = range_of(W, R, unit_start + tiles_b - 1);
+        for (int32_t r = r_lo; r <= r_hi; ++r) {
+            const int64_t slot = (int64_t)r + b * kHkv + g;
+            add(p.part_lse + slot * kGroup, p.part_o + slot * kGroup * kD);
+        }
+    }
+    // prefix pass
+    const int32_t i = c.seq_group[b];
+    if (i >= 0 && c.tok_offset[b] > 0) {
+        const int32_t t_i = c.ptiles_prefix[i + 1] - c.ptiles_prefix[i];
+        const int32_t b0 = c.group_start[i];
+        const int32_t n = min(c.group_start[i + 1] - b0, kMaxShare);
+        const int32_t W = c.chdr[kHdrTotalTiles], R = c.chdr[kHdrNumRanges];
+        const int32_t start = kHkv * c.ptiles_prefix[i] + g * t_i;
+        const int32_t splits = range_of(W, R, start + t_i - 1) - range_of(W, R, start) + 1;
+        const int64_t row0 = c.unit_rowbase[i * kHkv + g] + (b - b0);
+        for (int32_t s = 0; s < splits; ++s) {
+            const int64_t row = row0 + (int64_t)s * n;
+            add(c.pre_lse + row * kGroup, c.pre_o + row * kGroup * kD);
+        }
+    }
+    const int64_t row0 = (int64_t)b * kHq + g * kGroup;
+    #pragma unroll
+    for (int h = 0; h < kGroup; ++h) {
+        const bool any = z[h] > 0.f;
+        p.out[(row0 + h) * kD + d] = __float2bfloat16_rn(any ? acc[h] / z[h] : 0.f);
+        if (d == 0) p.lse[row0 + h] = any ? (mx[h] + log2f(z[h])) * 0.6931471805599453f : -INFINITY;
+    }
+}
+
+cudaError_t launch_combine_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
+    combine_cascade_kernel<<<p.batch * kHkv, kCombineThreads, 0, stream>>>(p, c);
+    return cudaGetLastError();
+}
+
+}  // namespace concur

@@ -59,6 +59,28 @@ struct DecodeParams {
     float* part_o;            // [2 * max_ranges][kGroup][kD] normalised partial outputs
     float* part_lse;          // [2 * max_ranges][kGroup]     base-2 log-sum-exp of each partial
     int32_t* unit_done;       // [batch * kHkv] partial segments finished per (sequence, KV head) unit
+    // shared-prefix (cascade) mode; both unset in the plain path
+    const int32_t* tok_offset; // [batch] first token of each sequence that this pass covers (multiple of 64), or null
+    int32_t all_partial;      // 1: every segment writes a partial into slot r + u (u = b * kHkv + g)
+};
+
+constexpr int kMaxShare = 10;     // siblings of a group that share one read of their common prefix
+
+// Shared-prefix (cascade) decode: groups of consecutive sequences whose first tokens are the
+// same cached pages.  Device pointers.
+struct CascadeParams {
+    const int32_t* group_start;   // [num_groups + 1] first sequence of each group; last entry = batch
+    const int32_t* prefix_lens;   // [num_groups] tokens the group's sequences have in common
+    int32_t num_groups;
+    int32_t max_rows;             // capacity of pre_o / pre_lse in (sibling, KV head) rows
+    int32_t grid_ctas;
+    int32_t* chdr;                // [kHdrWords] W', R', claim counter of the prefix pass
+    int32_t* tok_offset;          // [batch] shared tokens handled by the prefix pass (0 if none)
+    int32_t* seq_group;           // [batch] group of each sequence
+    int32_t* ptiles_prefix;       // [num_groups + 1] exclusive prefix of shared tiles per group
+    int32_t* unit_rowbase;        // [num_groups * kHkv + 1] first partial row of each prefix unit
+    float* pre_o;                 // [max_rows][kGroup][kD] normalised partials of the prefix pass
+    float* pre_lse;               // [max_rows][kGroup]     their base-2 log-sum-exp
 };
 
 // First flat tile of range r when [0, W) is cut into R ranges of equal size.
@@ -105,7 +127,8 @@ __device__ __forceinline__ int32_t find_range(const int32_t* __restrict__ range_
 
 // Segment of range r that starts at flat tile x (range_start[r] <= x < range_start[r+1]).
 __device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix, int32_t batch,
-                                              int32_t r, int32_t x0, int32_t x1, int32_t x) {
+                                              int32_t r, int32_t x0, int32_t x1, int32_t x,
+                                              int32_t all_partial = 0) {
     Segment s;
     s.b = find_sequence(prefix, batch, x);
     int32_t base = kHkv * prefix[s.b];
@@ -118,6 +141,9 @@ __device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix
     s.tile1 = end - unit_start;
     bool whole = (s.tile0 == 0) && (s.tile1 == s.tiles_b);
     s.slot = whole ? -1 : 2 * r + (x > x0 ? 1 : 0);
+    // cascade mode: every segment is a partial; (range, unit) pairs grow strictly along the flat
+    // tile space, so r + u is a unique slot below R + batch * kHkv
+    if (all_partial) s.slot = r + s.b * kHkv + s.g;
     return s;
 }
 
@@ -126,6 +152,9 @@ cudaError_t launch_plan(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_partial_scalar(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream);
+cudaError_t launch_plan_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
+cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
+cudaError_t launch_combine_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 int partial_scalar_ctas_per_sm();
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                           const int32_t* block_table, int32_t* seq_lens, int32_t* hdr, int32_t batch,

@@ -46,13 +46,15 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
         const int32_t x0 = p.range_start[r], x1 = p.range_start[r + 1];
         int32_t x = x0;
         while (x < x1) {
-            const Segment sg = segment_at(p.tiles_prefix, p.batch, r, x0, x1, x);
+            const Segment sg = segment_at(p.tiles_prefix, p.batch, r, x0, x1, x, p.all_partial);
             x += sg.tile1 - sg.tile0;
 
             int64_t n = p.seq_lens[sg.b];
             n = n < 0 ? 0 : (n > max_len ? max_len : n);
-            const int32_t tok0 = sg.tile0 * kTile;
-            const int32_t tok1 = (int32_t)min((int64_t)sg.tile1 * kTile, n);
+            // cascade mode: the first `off` tokens (a multiple of 64) belong to the prefix pass
+            const int32_t off = p.tok_offset ? p.tok_offset[sg.b] : 0;
+            const int32_t tok0 = off + sg.tile0 * kTile;
+            const int32_t tok1 = (int32_t)min((int64_t)off + (int64_t)sg.tile1 * kTile, n);
 
             // this lane's 8-wide piece of the 8 query rows, pre-scaled into the base-2 domain
             float q[kGroup][8];

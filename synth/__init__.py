@@ -237,3 +237,84 @@ def gather_sequences(w: Workload, seqs) -> Workload:
     return Workload(spec=sub, q=w.q[seqs].cpu(), k_pages=k, v_pages=v,
                     block_table=torch.from_numpy(table), seq_lens=torch.from_numpy(lens.astype(np.int32)),
                     scale=w.scale, lens_host=lens.astype(np.int32), table_host=table)
+
+
+@dataclass
+class CascadeWorkload:
+    """A workload whose sequences come in groups of siblings that share their first tokens'
+    pages (the samples drawn for one prompt)."""
+    w: Workload
+    group_start: torch.Tensor      # [G + 1] int32
+    prefix_lens: torch.Tensor      # [G] int32: tokens whose pages the group's sequences share
+    group_start_host: np.ndarray = field(default=None)
+    prefix_lens_host: np.ndarray = field(default=None)
+
+    def logical_bytes(self) -> int:
+        """Algorithmic bytes if every sequence read its whole context itself."""
+        return self.w.algorithmic_bytes()
+
+    def shared_bytes(self) -> int:
+        """Algorithmic bytes when the shared pages of a group are counted once."""
+        s = self.w.spec
+        per_token = 2 * s.num_kv_heads * s.head_dim * 2
+        saved = 0
+        for i, pre in enumerate(self.prefix_lens_host):
+            n = int(self.group_start_host[i + 1] - self.group_start_host[i])
+            saved += (n - 1) * int(pre) * per_token
+        return self.w.algorithmic_bytes() - saved
+
+
+def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0) -> CascadeWorkload:
+    """groups: list of (shared_tokens, [own_tokens of each sibling]).  `shared_tokens` must be a
+    multiple of the page size (only whole pages can be shared physically).  Sequence lengths are
+    shared + own; siblings point at the same physical pages for the shared part; all pages are
+    shuffled in one seeded permutation; values are i.i.d. N(0,1) (q: N(0, q_std^2))."""
+    P = page_size
+    lens, gstart, pre = [], [0], []
+    for shared, owns in groups:
+        assert shared % P == 0 and len(owns) >= 1
+        lens += [shared + int(o) for o in owns]
+        gstart.append(len(lens))
+        pre.append(shared)
+    lens = np.asarray(lens, dtype=np.int32)
+    spec = Spec(name, len(lens), P, ("list", [int(x) for x in lens]), seed=seed, q_std=q_std)
+    # page allocation: shared pages once per group, then each sibling's own pages
+    rows, total = [], 0
+    for (shared, owns), b0 in zip(groups, gstart[:-1]):
+        shared_pages = list(range(total, total + shared // P))
+        total += shared // P
+        for j, o in enumerate(owns):
+            n_own = (shared + int(o) + P - 1) // P - shared // P
+            rows.append(shared_pages + list(range(total, total + n_own)))
+            total += n_own
+    num_pages = max(total, 1)
+    perm = _rng(seed, 2).permutation(num_pages)
+    width = max(1, max(len(r) for r in rows))
+    table = np.full((len(lens), width), -1, dtype=np.int32)
+    for b, r in enumerate(rows):
+        table[b, :len(r)] = perm[np.asarray(r, dtype=np.int64)] if r else []
+    device = torch.device(device)
+
+    def gen(stream):
+        g = torch.Generator(device=device)
+        g.manual_seed(seed * 1000 + stream)
+        return g
+
+    Hq, Hkv, D = spec.num_q_heads, spec.num_kv_heads, spec.head_dim
+    q = _normal_bf16((spec.batch, Hq, D), q_std, gen(3), device)
+    k = _normal_bf16((num_pages, Hkv, P, D), 1.0, gen(4), device)
+    v = _normal_bf16((num_pages, Hkv, P, D), 1.0, gen(5), device)
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16, device=device)
+    for b, n in enumerate(lens):
+        n = int(n)
+        if n % P:
+            page = int(table[b, (n - 1) // P])
+            k[page, :, n % P:, :] = nan
+            v[page, :, n % P:, :] = nan
+    w = Workload(spec=spec, q=q, k_pages=k, v_pages=v, block_table=torch.from_numpy(table).to(device),
+                 seq_lens=torch.from_numpy(lens).to(device),
+                 scale=float(np.float32(1.0) / np.sqrt(np.float32(D))), lens_host=lens, table_host=table)
+    gs = np.asarray(gstart, dtype=np.int32)
+    pl = np.asarray(pre, dtype=np.int32)
+    return CascadeWorkload(w=w, group_start=torch.from_numpy(gs).to(device), prefix_lens=torch.from_numpy(pl).to(device),
+                           group_start_host=gs, prefix_lens_host=pl)
