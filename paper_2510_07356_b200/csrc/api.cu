@@ -203,7 +203,7 @@ int concur_decode_attn(concur_attn_t* h, const void* q, const void* k_pages, con
     if (rc != CONCUR_OK || batch == 0) return rc;
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok()) return CONCUR_ERR_CUDA;
-    DecodeParams p;
+    DecodeParams p = {};
     fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
                 block_table_stride);
     return enqueue(h, p, static_cast<cudaStream_t>(cuda_stream));
@@ -277,7 +277,7 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
     if ((rc = ensure(h->cascade_ws, lay.total)) != CONCUR_OK) return rc;
     char* cw = static_cast<char*>(h->cascade_ws.ptr);
 
-    DecodeParams p;
+    DecodeParams p = {};
     fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
                 block_table_stride);
     CascadeParams c;
@@ -345,7 +345,7 @@ int concur_decode_attn_host(concur_attn_t* h, const void* q, const void* k_pages
     ok &= cudaMemcpyAsync(h->st_bt.ptr, block_table, bt_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     ok &= cudaMemcpyAsync(h->st_len.ptr, seq_lens, len_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return CONCUR_ERR_CUDA; }
-    DecodeParams p;
+    DecodeParams p = {};
     fill_params(h, p, h->st_q.ptr, h->st_k.ptr, h->st_v.ptr, static_cast<const int32_t*>(h->st_bt.ptr),
                 static_cast<const int32_t*>(h->st_len.ptr), scale, h->st_out.ptr,
                 static_cast<float*>(h->st_lse.ptr), batch, num_pages, block_table_stride);

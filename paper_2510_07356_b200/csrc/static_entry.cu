@@ -90,7 +90,7 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     int rc = setup_current_device(dev, &s);
     if (rc != CONCUR_OK) return rc;
 
-    DecodeParams p;
+    DecodeParams p = {};
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.k_pages = static_cast<const __nv_bfloat16*>(k_pages);
     p.v_pages = static_cast<const __nv_bfloat16*>(v_pages);
