@@ -77,6 +77,9 @@ typedef enum {
 #define CONCUR_OPT_CLAIM_AHEAD  9   /* tiles before a range's end at which a CTA claims its next range
                                        (default: at the range's first tile)                              */
 
+#define CONCUR_OPT_PREFIX_KERNEL 10 /* shared-prefix pass of the cascade step: 0 (default) = tcgen05 kernel with
+                                       TMEM accumulators, 1 = warp-level mma.sync kernel                 */
+
 typedef struct concur_attn concur_attn_t;   /* opaque; owns its workspace and nothing else */
 
 typedef struct {

@@ -31,6 +31,7 @@ CONCUR_OPT_EVENT_BEFORE_PARTIAL = 6
 CONCUR_OPT_EVENT_AFTER_PARTIAL = 7
 CONCUR_OPT_FUSE_COMBINE = 8
 CONCUR_OPT_CLAIM_AHEAD = 9
+CONCUR_OPT_PREFIX_KERNEL = 10
 
 EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",

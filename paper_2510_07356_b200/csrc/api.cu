@@ -83,6 +83,7 @@ struct concur_attn {
     int32_t min_range_tiles = 0;
     int32_t fuse_combine = 1;
     int32_t claim_ahead = 1 << 20;
+    int32_t prefix_kernel = 0;
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;
     Staging st_q, st_k, st_v, st_bt, st_len, st_out, st_lse;
     Staging cascade_ws;          // allocated on the first cascade call
@@ -302,7 +303,8 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (launch_plan_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
-    if (launch_prefix_mma(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    if ((h->prefix_kernel == 1 ? launch_prefix_mma(p, c, stream) : launch_prefix_tc(p, c, stream)) != cudaSuccess)
+        return CONCUR_ERR_CUDA;
     cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream);
     if (e != cudaSuccess) return CONCUR_ERR_CUDA;
     if (launch_combine_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
@@ -399,6 +401,9 @@ int concur_attn_set_option(concur_attn_t* h, int32_t key, int64_t value) {
         case CONCUR_OPT_CLAIM_AHEAD:
             if (value > (1 << 20)) return CONCUR_ERR_INVALID_ARG;
             h->claim_ahead = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_PREFIX_KERNEL:
+            if (value > 1) return CONCUR_ERR_INVALID_ARG;
+            h->prefix_kernel = (int32_t)value; return CONCUR_OK;
         case CONCUR_OPT_EVENT_BEFORE_PARTIAL:
             h->ev_before = reinterpret_cast<cudaEvent_t>(static_cast<uintptr_t>(value)); return CONCUR_OK;
         case CONCUR_OPT_EVENT_AFTER_PARTIAL:

@@ -18,11 +18,12 @@ def P():
     return pkg
 
 
-def run_cascade(P, cw, prefix_lens=None, kernel=0, ranges=0):
+def run_cascade(P, cw, prefix_lens=None, kernel=0, ranges=0, prefix_kernel=0):
     w = cw.w
     attn = P.DecodeAttention(w.spec.page_size, w.spec.batch, w.block_table.shape[1], 0)
     attn.set_option(P.CONCUR_OPT_KERNEL, kernel)
     attn.set_option(P.CONCUR_OPT_NUM_RANGES, ranges)
+    attn.set_option(P.CONCUR_OPT_PREFIX_KERNEL, prefix_kernel)
     out = torch.full_like(w.q, 7.0)
     lse = torch.full((w.spec.batch, 64), 7.0, dtype=torch.float32, device="cuda:0")
     pl = cw.prefix_lens if prefix_lens is None else prefix_lens
@@ -45,14 +46,16 @@ GROUPS = [
 ]
 
 
-@pytest.mark.parametrize("page_size", [16, 64])
+@pytest.mark.parametrize("page_size", [16, 32, 64])
 @pytest.mark.parametrize("kernel", [0, 1])
-def test_cascade_matches_oracle(P, page_size, kernel):
+@pytest.mark.parametrize("prefix_kernel", [0, 1])
+def test_cascade_matches_oracle(P, page_size, kernel, prefix_kernel):
+    """prefix_kernel 0: tcgen05 / TMEM prefix pass; 1: warp-level mma.sync prefix pass."""
     cw = synth.make_cascade_workload(f"casc_p{page_size}", GROUPS, page_size, 4000 + page_size, "cuda:0")
-    out, lse, attn = run_cascade(P, cw, kernel=kernel)
+    out, lse, attn = run_cascade(P, cw, kernel=kernel, prefix_kernel=prefix_kernel)
     assert attn.status() == 0
     ref_out, ref_lse = oracle_sequences(synth.gather_sequences(cw.w, range(cw.w.spec.batch)))
-    assert_parity(out, lse, ref_out, ref_lse, f"cascade p{page_size} kernel {kernel}")
+    assert_parity(out, lse, ref_out, ref_lse, f"cascade p{page_size} kernel {kernel} prefix kernel {prefix_kernel}")
     attn.close()
 
 
@@ -91,6 +94,9 @@ def test_long_shared_prefix_split_over_many_ctas(P):
         out, lse, a2 = run_cascade(P, cw, ranges=ranges)
         assert_parity(out, lse, ref_out, ref_lse, f"long shared prefix, {ranges} suffix ranges")
         a2.close()
+    out, lse, a3 = run_cascade(P, cw, prefix_kernel=1)
+    assert_parity(out, lse, ref_out, ref_lse, "long shared prefix, mma.sync prefix pass")
+    a3.close()
     attn.close()
 
 
