@@ -7,19 +7,39 @@
 // one place of the decode step that is a dense contraction (80 flop per KV byte at ten
 // siblings), so it runs on tcgen05 with its accumulators in tensor memory:
 //
-//   S[128 x 64]   = Q[128 x 128] . K_tile^T            (8 MMAs of K = 16; S in TMEM, double-buffered)
+//   S[128 x 64]   = Q[128 x 128] . K_tile^T            (8 MMAs of K = 16; S in TMEM)
 //   online softmax, one thread per row: thread t owns TMEM lane t = (sibling t / 8, head t % 8);
-//                 it reads its 64 scores with one tcgen05.ld, keeps the running maximum and sum in
-//                 registers, and writes P = 2^(S - m) as bf16 into a swizzled shared-memory tile
+//                 it reads its 64 scores with tcgen05.ld, keeps the reference maximum and the sum
+//                 in registers, and writes P = 2^(S - m) as packed bf16 back into TMEM
 //   O[128 x 128] += P[128 x 64] . V_tile[64 x 128]     (4 MMAs of K = 16; O in TMEM, V is the
 //                 MN-major B operand exactly as TMA laid it down)
-//   when a row's maximum moves, its O row is rescaled in TMEM (tcgen05.ld / st) before the
-//   next P.V product is released.
 //
-// Warp roles: warps 0-3 softmax / rescale / epilogue (128 threads = 128 TMEM lanes), warp 4
-// TMA producer, warp 5 issues the MMAs (one thread) and owns the TMEM allocation.  The MMA
-// thread issues Q.K^T of tile i + 1 before P.V of tile i, so the tensor pipe works on the next
-// scores while the softmax threads are busy with the current ones.
+// Both A operands live in TMEM: the queries are copied there once per segment (they do not
+// change from tile to tile) and P never leaves it, so the only shared-memory traffic of the
+// tensor pipe is one pass over the K tile and one over the V tile.  (With Q and P as
+// shared-memory operands the pipe spent ~1,100 clocks per tile fetching them -- more than the
+// HBM time of the tile.)
+//
+// One softmax warp per SM sub-partition is a serial chain (TMEM load, maximum, 64 exponentials
+// at 4 per clock, pack, store, fences) of about 1,900 clocks per tile, which is below the HBM
+// rate.  So there are TWO softmax warpgroups that take alternate tiles, each with its own
+// score buffer, P columns and O accumulator (TMEM columns: Q, S_A, S_B, P_A, P_B, O_A, O_B); while one group
+// is in its exponentials the other loads its scores.  At the end of a segment the two
+// (m, l, O) states of every row are merged by their log-sum-exp, each group writing half of
+// the output columns.
+//
+// A row's O is rescaled in TMEM (tcgen05.ld / st) only when a tile raises its maximum by more
+// than a fixed slack over the reference its probabilities are scaled with, so in the steady
+// state the softmax threads never touch O.
+//
+// Warp roles: warps 0-3 softmax group A, warps 4-7 softmax group B (a warp may touch the TMEM
+// lanes 32 (w % 4) .. + 31), warp 8 TMA producer, warp 9 issues the Q.K^T MMAs (one thread) and
+// owns the TMEM allocation, warp 10 issues the P.V MMAs.  One issuing thread for both was the
+// bottleneck (about 90 clocks per tcgen05.mma and as much again in barrier waits and commits,
+// all serial); the two products depend on different events (K landed and score buffer read,
+// against P written and V landed), so each gets its own thread.  Q.K^T of tile i is issued
+// as soon as the score buffer of tile i - 2 has been read, so a group's next scores are ready
+// when it finishes a tile.
 //
 // Input / output contract is that of the plan: a segment (the part of a unit inside one range)
 // ends with one normalised fp32 partial (out, base-2 lse) per sibling in rows `row .. row + n`
@@ -37,49 +57,54 @@ namespace concur {
 
 namespace {
 
-constexpr int kTStages = 5;
-constexpr int kTProducerWarp = 4;
-constexpr int kTMmaWarp = 5;
-constexpr int kTThreads = 6 * 32;
+constexpr int kTKStages = 5;                              // K ring: a stage is free again after Q.K^T
+constexpr int kTVStages = 6;                              // V ring: a stage is free again after P.V
+constexpr int kTVLag = 2;                                 // V of tile t is requested with K of tile t + 2
+constexpr int kTMetaRing = 16;                            // tile records; readers trail the producer by < 8
+constexpr int kTProducerWarp = 8;
+constexpr int kTMmaWarp = 9;                              // issues Q.K^T, owns the TMEM allocation
+constexpr int kTPvWarp = 10;                              // issues P.V
+constexpr int kTThreads = 11 * 32;
 constexpr int kTRows = 128;                               // MMA M
 constexpr int kTHalfBytes = kTile * 128;                  // 8 KB: 64 tokens x one 64-dim half
 constexpr int kTTileBytes = 2 * kTHalfBytes;              // 16 KB: one K or V tile
-constexpr int kTStageBytes = 2 * kTTileBytes;             // K | V
 constexpr int kTQRows = kMaxShare * kGroup;               // 80 query rows that are really loaded
 constexpr int kTQHalfBytes = kTQRows * 128;               // 10 KB
 constexpr int kTQBytes = 2 * kTQHalfBytes;                // 20 KB per buffer
-constexpr int kTPBytes = kTRows * 128;                    // 16 KB: P tile, 128 rows x 64 tokens bf16
-constexpr uint32_t kTmemCols = 256;                       // S0 [0,64)  S1 [64,128)  O [128,256)
-constexpr uint32_t kTmemO = 128;
+// TMEM columns (512): Q as packed bf16 [0,64); S_A [64,128), S_B [128,192); P_A [192,224),
+// P_B [224,256) as packed bf16; O_A [256,384), O_B [384,512)
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemQ = 0, kTmemS = 64, kTmemP = 192, kTmemO = 256;
 
 static_assert(kTQHalfBytes % 1024 == 0, "query halves must keep the swizzle phase");
 
 struct TMeta {
     int32_t n;            // sharing siblings (2..kMaxShare); 0 = no more work
-    int32_t first, last;  // first / last tile of its segment
+    int32_t idx, cnt;     // index of the tile in its segment, tiles of the segment
     int32_t qsel;         // query buffer of the segment
     int32_t row;          // first partial row of the segment (one row per sibling)
-    int32_t pad[3];
+    int32_t g;            // KV head
+    int32_t pages[4];     // physical pages of the tile (64 / P of them)
+    int32_t pad[6];
 };
+static_assert(sizeof(TMeta) == 64, "one record per 64 bytes");
 
-// Shared memory, from a 1024-byte aligned base.  The MMA reads 128 A rows; the query buffers
-// hold 80, so the rows beyond them alias whatever follows (the other query buffer, the P tile):
-// always inside this allocation, and only ever feeding accumulator rows that are not written out.
+// Shared memory, from a 1024-byte aligned base.
 struct TSmem {
-    static constexpr int kQOff = kTStages * kTStageBytes;                 // 2 x 20 KB
-    static constexpr int kPOff = kQOff + 2 * kTQBytes;                    // 16 KB
-    static constexpr int kMetaOff = kPOff + kTPBytes;
-    static constexpr int kBarOff = kMetaOff + kTStages * (int)sizeof(TMeta);
-    // full_k, full_v, empty per stage; q_full x2, q_empty x2; s_full x2, s_free x2; p_full; pv_done
-    static constexpr int kNumBars = 3 * kTStages + 10;
+    static constexpr int kVOff = kTKStages * kTTileBytes;
+    static constexpr int kQOff = kVOff + kTVStages * kTTileBytes;         // 2 x 20 KB staging of the queries
+    static constexpr int kXchOff = kQOff + 2 * kTQBytes;                  // [2 groups][128 rows] (m, l)
+    static constexpr int kMetaOff = kXchOff + 2 * kTRows * 8;
+    static constexpr int kBarOff = kMetaOff + kTMetaRing * (int)sizeof(TMeta);
+    // full_k, empty_k per K stage; full_v, empty_v per V stage; meta_full per record; then pairs:
+    // q_full, q_empty, s_full, s_free, p_full, pv_done; xch_a, xch_b; qt_ready, qt_free
+    static constexpr int kNumBars = 2 * kTKStages + 2 * kTVStages + kTMetaRing + 16;
     static constexpr int kTmemPtrOff = kBarOff + kNumBars * 8;
     static constexpr int kAbortOff = kTmemPtrOff + 8;
     static constexpr int kTotal = kAbortOff + 8;
     static constexpr int kBytes = kTotal + 1024;
 };
-static_assert(TSmem::kPOff % 1024 == 0 && TSmem::kQOff % 1024 == 0, "operand slabs must be 1024-byte aligned");
-static_assert(TSmem::kQOff + kTQBytes + kTQHalfBytes + kTRows * 128 <= TSmem::kPOff + kTPBytes,
-              "the 128-row view of the last query half must stay inside the allocation");
+static_assert(TSmem::kVOff % 1024 == 0 && TSmem::kQOff % 1024 == 0, "operand slabs must be 1024-byte aligned");
 static_assert(TSmem::kBytes <= 232448, "exceeds the 227 KB a CTA may use");
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, int32_t c2,
@@ -98,40 +123,50 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
     TMeta* meta = reinterpret_cast<TMeta*>(smem + TSmem::kMetaOff);
+    float2* xch = reinterpret_cast<float2*>(smem + TSmem::kXchOff);
     volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(smem + TSmem::kAbortOff);
     volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(smem + TSmem::kTmemPtrOff);
     const uint32_t bar_base = smem_base + TSmem::kBarOff;
+    constexpr int kB0 = 2 * kTKStages + 2 * kTVStages + kTMetaRing;
     auto full_k = [&](int s) { return bar_base + 8u * s; };
-    auto full_v = [&](int s) { return bar_base + 8u * (kTStages + s); };
-    auto empty = [&](int s) { return bar_base + 8u * (2 * kTStages + s); };
-    auto q_full = [&](int i) { return bar_base + 8u * (3 * kTStages + i); };
-    auto q_empty = [&](int i) { return bar_base + 8u * (3 * kTStages + 2 + i); };
-    auto s_full = [&](int i) { return bar_base + 8u * (3 * kTStages + 4 + i); };
-    auto s_free = [&](int i) { return bar_base + 8u * (3 * kTStages + 6 + i); };
-    const uint32_t p_full = bar_base + 8u * (3 * kTStages + 8);
-    const uint32_t pv_done = bar_base + 8u * (3 * kTStages + 9);
+    auto empty_k = [&](int s) { return bar_base + 8u * (kTKStages + s); };
+    auto full_v = [&](int s) { return bar_base + 8u * (2 * kTKStages + s); };
+    auto empty_v = [&](int s) { return bar_base + 8u * (2 * kTKStages + kTVStages + s); };
+    auto meta_full = [&](int s) { return bar_base + 8u * (2 * kTKStages + 2 * kTVStages + s); };
+    auto q_full = [&](int i) { return bar_base + 8u * (kB0 + i); };
+    auto q_empty = [&](int i) { return bar_base + 8u * (kB0 + 2 + i); };
+    auto s_full = [&](int i) { return bar_base + 8u * (kB0 + 4 + i); };
+    auto s_free = [&](int i) { return bar_base + 8u * (kB0 + 6 + i); };
+    auto p_full = [&](int i) { return bar_base + 8u * (kB0 + 8 + i); };
+    auto pv_done = [&](int i) { return bar_base + 8u * (kB0 + 10 + i); };
+    const uint32_t xch_a = bar_base + 8u * (kB0 + 12);               // both groups have published (m, l)
+    const uint32_t xch_b = xch_a + 8u;                               // both groups have read both O
+    const uint32_t qt_ready = xch_a + 16u;                           // the segment's queries are in TMEM
+    const uint32_t qt_free = xch_a + 24u;                            // the segment's last Q.K^T has completed
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int32_t P = p.page_size;
 
     // unused query rows must at least be defined once
-    for (int i = tid; i < (2 * kTQBytes + kTPBytes) / 16; i += kTThreads)
+    for (int i = tid; i < (2 * kTQBytes) / 16; i += kTThreads)
         reinterpret_cast<uint4*>(smem + TSmem::kQOff)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
-        for (int s = 0; s < kTStages; ++s) {
-            mbar_init(full_k(s), 1);
-            mbar_init(full_v(s), 1);
-            mbar_init(empty(s), 1);
-        }
+        for (int s = 0; s < kTKStages; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
+        for (int s = 0; s < kTVStages; ++s) { mbar_init(full_v(s), 1); mbar_init(empty_v(s), 1); }
+        for (int s = 0; s < kTMetaRing; ++s) mbar_init(meta_full(s), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(q_full(i), 1);
-            mbar_init(q_empty(i), 1);
+            mbar_init(q_empty(i), 128);
             mbar_init(s_full(i), 1);
             mbar_init(s_free(i), 128);
+            mbar_init(p_full(i), 128);
+            mbar_init(pv_done(i), 1);
         }
-        mbar_init(p_full, 128);
-        mbar_init(pv_done, 1);
+        mbar_init(xch_a, 256);
+        mbar_init(xch_b, 256);
+        mbar_init(qt_ready, 128);
+        mbar_init(qt_free, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -146,11 +181,28 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
 
     if (warp == kTProducerWarp) {
         // =========================================================== producer warp
-        uint32_t it = 0, seg = 0;
+        uint32_t it = 0, vt = 0, seg = 0;                      // K tiles, V tiles, segments issued
         bool ok = true;
         const int pages_per_tile_shift = 6 - p.page_shift;
         const int32_t npages = kTile >> p.page_shift;
         const uint32_t page_bytes = (uint32_t)P * 128u;        // one half of one page
+        // V of tile u (lane 0 only): its pages are still in the tile's record
+        auto issue_v = [&](uint32_t u) {
+            const TMeta& m = meta[u % kTMetaRing];
+            const int vs = u % kTVStages;
+            ok = mbar_wait(empty_v(vs), ((u / kTVStages) & 1u) ^ 1u, abort_flag);
+            if (!ok) return;
+            const uint32_t vdst = smem_base + TSmem::kVOff + vs * kTTileBytes;
+            mbar_arrive_expect_tx(full_v(vs), kTTileBytes);
+            #pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (q < npages) {
+                    const int32_t prow = (m.pages[q] * kHkv + m.g) * P;
+                    tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(vs));
+                    tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(vs));
+                }
+            ++vt;
+        };
         int32_t r = blockIdx.x;
         while (ok && r < R) {
             int32_t r_next = 0;
@@ -184,8 +236,7 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                         pg = pg_next;
                         pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                     }
-                    const int s = it % kTStages;
-                    const uint32_t parity = (it / kTStages) & 1u;
+                    const int ks = it % kTKStages;
                     int32_t my_page = __shfl_sync(0xffffffffu, pg, (first_page - chunk_base + (lane & 3)) & 31);
                     const bool bad = (lane < npages) && (my_page < 0 || my_page >= p.num_pages);
                     if (__any_sync(0xffffffffu, bad)) {
@@ -208,28 +259,22 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                                 }
                             }
                         }
-                        if (ok) ok = mbar_wait(empty(s), parity ^ 1u, abort_flag);
+                        if (ok) ok = mbar_wait(empty_k(ks), ((it / kTKStages) & 1u) ^ 1u, abort_flag);
                         if (ok) {
-                            TMeta& m = meta[s];
-                            m.n = n; m.first = (t == tile0); m.last = (t == tile1 - 1); m.qsel = qsel; m.row = row;
-                            const uint32_t kdst = smem_base + s * kTStageBytes;
-                            const uint32_t vdst = kdst + kTTileBytes;
-                            mbar_arrive_expect_tx(full_k(s), kTTileBytes);
+                            TMeta& m = meta[it % kTMetaRing];
+                            m.n = n; m.idx = t - tile0; m.cnt = tile1 - tile0; m.qsel = qsel; m.row = row; m.g = g;
+                            m.pages[0] = pages[0]; m.pages[1] = pages[1]; m.pages[2] = pages[2]; m.pages[3] = pages[3];
+                            mbar_arrive(meta_full(it % kTMetaRing));
+                            const uint32_t kdst = smem_base + ks * kTTileBytes;
+                            mbar_arrive_expect_tx(full_k(ks), kTTileBytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
                                 if (q < npages) {
                                     const int32_t prow = (pages[q] * kHkv + g) * P;
-                                    tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(s));
-                                    tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(s));
+                                    tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
+                                    tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
                                 }
-                            mbar_arrive_expect_tx(full_v(s), kTTileBytes);
-                            #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                if (q < npages) {
-                                    const int32_t prow = (pages[q] * kHkv + g) * P;
-                                    tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(s));
-                                    tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(s));
-                                }
+                            if (it >= (uint32_t)kTVLag) issue_v(it - kTVLag);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -240,183 +285,266 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
             r = __shfl_sync(0xffffffffu, r_next, 0);
         }
         if (lane == 0) {
+            while (ok && vt < it) issue_v(vt);                 // the last tiles' V
             if (ok) {
-                const int s = it % kTStages;
-                ok = mbar_wait(empty(s), ((it / kTStages) & 1u) ^ 1u, abort_flag);
-                if (ok) { meta[s].n = 0; mbar_arrive(full_k(s)); }
+                meta[it % kTMetaRing].n = 0;                   // no more work
+                mbar_arrive(meta_full(it % kTMetaRing));
             }
             if (!ok) {
                 wait_failed(p, abort_flag, 31);
                 // let the copies still in flight land before the CTA's shared memory is released
-                const uint32_t lo = it > (uint32_t)kTStages ? it - kTStages : 0u;
-                for (uint32_t j = lo; j < it; ++j) {
-                    volatile int32_t never = 0;
-                    mbar_wait(full_k(j % kTStages), (j / kTStages) & 1u, &never);
-                    mbar_wait(full_v(j % kTStages), (j / kTStages) & 1u, &never);
-                }
+                volatile int32_t never = 0;
+                for (uint32_t j = it > (uint32_t)kTKStages ? it - kTKStages : 0u; j < it; ++j)
+                    mbar_wait(full_k(j % kTKStages), (j / kTKStages) & 1u, &never);
+                for (uint32_t j = vt > (uint32_t)kTVStages ? vt - kTVStages : 0u; j < vt; ++j)
+                    mbar_wait(full_v(j % kTVStages), (j / kTVStages) & 1u, &never);
             }
         }
     } else if (warp == kTMmaWarp) {
-        // =========================================================== MMA warp (one thread issues)
+        // =========================================================== Q.K^T warp (one thread issues)
         if (lane == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kTRows, kTile, false, false);
-            constexpr uint32_t idesc_pv = umma_idesc_bf16(kTRows, kD, false, true);
-            const uint32_t p_addr = smem_base + TSmem::kPOff;
-            bool ok = true, have_prev = false;
-            int ps = 0;
-            uint32_t pparity = 0, pfirst = 0, segs = 0;
+            bool ok = true;
             int site = 0;
+            uint32_t segs = 0;
             for (uint32_t it = 0; ok; ++it) {
-                const int s = it % kTStages;
-                const uint32_t parity = (it / kTStages) & 1u;
-                if (!mbar_wait(full_k(s), parity, abort_flag)) { ok = false; site = 32; break; }
-                const TMeta mt = meta[s];
-                const bool done = (mt.n == 0);
-                auto issue_qk = [&]() {
-                    if (mt.first) {
-                        if (!mbar_wait(q_full(mt.qsel), (segs >> 1) & 1u, abort_flag)) { ok = false; site = 33; return; }
-                        ++segs;
-                    }
-                    const int sb = it & 1u;
-                    if (!mbar_wait(s_free(sb), ((it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; site = 34; return; }
-                    tc_fence_after_sync();
-                    const uint32_t q_addr = smem_base + TSmem::kQOff + mt.qsel * kTQBytes;
-                    const uint32_t k_addr = smem_base + s * kTStageBytes;
-                    #pragma unroll
-                    for (int k16 = 0; k16 < 8; ++k16) {
-                        const uint32_t koff = (uint32_t)(k16 & 3) * 32u;
-                        const uint64_t a = umma_smem_desc(q_addr + (k16 >> 2) * kTQHalfBytes + koff, 16, 1024);
-                        const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
-                        umma_ss(tmem_base + sb * kTile, a, b, idesc_qk, k16 > 0);
-                    }
-                    umma_commit(s_full(sb));
-                    if (mt.last) umma_commit(q_empty(mt.qsel));      // the segment's last read of its query buffer
-                };
-                auto issue_pv = [&]() {
-                    if (!mbar_wait(p_full, (it - 1) & 1u, abort_flag)) { ok = false; site = 35; return; }
-                    if (!mbar_wait(full_v(ps), pparity, abort_flag)) { ok = false; site = 36; return; }
-                    tc_fence_after_sync();
-                    const uint32_t v_addr = smem_base + ps * kTStageBytes + kTTileBytes;
-                    #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t a = umma_smem_desc(p_addr + kk * 32, 16, 1024);
-                        const uint64_t b = umma_smem_desc(v_addr + kk * 2048, kTHalfBytes, 1024);
-                        umma_ss(tmem_base + kTmemO, a, b, idesc_pv, (pfirst && kk == 0) ? 0u : 1u);
-                    }
-                    umma_commit(empty(ps));          // K and V of that stage may be overwritten
-                    umma_commit(pv_done);
-                };
-                // scores of tile `it` first, so that they are computed while the softmax threads
-                // work on tile it - 1; at a segment start the new queries may still be in flight,
-                // so the pending P.V goes first there
-                if (!done && !mt.first) issue_qk();
-                if (ok && have_prev) issue_pv();
-                if (ok && !done && mt.first) issue_qk();
-                if (done) break;
-                have_prev = true; ps = s; pparity = parity; pfirst = mt.first;
+                const int g = it & 1u;
+                if (!mbar_wait(meta_full(it % kTMetaRing), (it / kTMetaRing) & 1u, abort_flag)) { ok = false; site = 32; break; }
+                const TMeta mt = meta[it % kTMetaRing];
+                if (mt.n == 0) break;
+                const int ks = it % kTKStages;
+                if (!mbar_wait(full_k(ks), (it / kTKStages) & 1u, abort_flag)) { ok = false; site = 43; break; }
+                if (mt.idx == 0) {                            // a segment starts: its queries must be in TMEM
+                    if (!mbar_wait(qt_ready, segs & 1u, abort_flag)) { ok = false; site = 33; break; }
+                    ++segs;
+                }
+                // the group has copied the scores of its previous tile out of the buffer
+                if (!mbar_wait(s_free(g), ((it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; site = 34; break; }
+                tc_fence_after_sync();
+                const uint32_t k_addr = smem_base + ks * kTTileBytes;
+                #pragma unroll
+                for (int k16 = 0; k16 < 8; ++k16) {
+                    const uint32_t koff = (uint32_t)(k16 & 3) * 32u;
+                    const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
+                    umma_ts(tmem_base + kTmemS + g * kTile, tmem_base + kTmemQ + k16 * 8, b, idesc_qk, k16 > 0);
+                }
+                umma_commit(s_full(g));
+                umma_commit(empty_k(ks));                                   // that K stage may be overwritten
+                if (mt.idx == mt.cnt - 1) umma_commit(qt_free);            // the segment's last read of its queries
+            }
+            if (!ok) wait_failed(p, abort_flag, site);
+        }
+        __syncwarp();
+    } else if (warp == kTPvWarp) {
+        // =========================================================== P.V warp (one thread issues)
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = umma_idesc_bf16(kTRows, kD, false, true);
+            bool ok = true;
+            int site = 0;
+            for (uint32_t u = 0; ok; ++u) {
+                const int g = u & 1u;
+                if (!mbar_wait(meta_full(u % kTMetaRing), (u / kTMetaRing) & 1u, abort_flag)) { ok = false; site = 46; break; }
+                const TMeta mt = meta[u % kTMetaRing];
+                if (mt.n == 0) break;
+                const int vs = u % kTVStages;
+                if (!mbar_wait(p_full(g), (u >> 1) & 1u, abort_flag)) { ok = false; site = 35; break; }
+                if (!mbar_wait(full_v(vs), (u / kTVStages) & 1u, abort_flag)) { ok = false; site = 36; break; }
+                tc_fence_after_sync();
+                const uint32_t v_addr = smem_base + TSmem::kVOff + vs * kTTileBytes;
+                #pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t b = umma_smem_desc(v_addr + kk * 2048, kTHalfBytes, 1024);
+                    // a group's first tile of a segment overwrites its accumulator
+                    umma_ts(tmem_base + kTmemO + g * kD, tmem_base + kTmemP + g * 32 + kk * 8, b, idesc_pv,
+                            (mt.idx < 2 && kk == 0) ? 0u : 1u);
+                }
+                umma_commit(empty_v(vs));               // that V stage may be overwritten
+                umma_commit(pv_done(g));
             }
             if (!ok) wait_failed(p, abort_flag, site);
         }
         __syncwarp();
     } else {
         // =========================================================== softmax warps (thread = row)
-        const int j = tid >> 3, head = tid & 7;                  // sibling, head of this row
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const uint32_t p_row = smem_base + TSmem::kPOff + (uint32_t)tid * 128u;
-        const int sw = tid & 7;
-        float m = -INFINITY, l = 0.f;
+        const int g = warp >> 2;                                 // group: tiles with (it & 1) == g
+        const int row = tid & 127;
+        const int j = row >> 3, head = row & 7;                  // sibling, head of this row
+        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t o_mine = lane_base + kTmemO + g * kD, o_other = lane_base + kTmemO + (g ^ 1) * kD;
+        const int sw = row & 7;
+        const float sc = p.scale_log2e;
+        const bool sc_neg = sc < 0.f;
+        // The scale used for a row's probabilities is 2^-m_ref, where m_ref trails the true running
+        // maximum by at most kSlack (in base-2 units): P stays below 2^kSlack, which bf16 and the
+        // fp32 sums hold without loss, and O has to be rescaled in TMEM only when a tile raises
+        // the maximum by more than that -- a handful of times per segment instead of per tile.
+        constexpr float kSlack = 8.f;
+        float m_ref = -INFINITY, l = 0.f;
+        uint32_t k = 0, segs = 0, qsegs = 0;                     // tiles this group has taken; segments ended / started
         bool ok = true;
         int site = 0;
         for (uint32_t it = 0; ok; ++it) {
-            const int s = it % kTStages;
-            const uint32_t parity = (it / kTStages) & 1u;
-            if (!mbar_wait(full_k(s), parity, abort_flag)) { ok = false; site = 37; break; }
-            const TMeta mt = meta[s];
+            if (!mbar_wait(meta_full(it % kTMetaRing), (it / kTMetaRing) & 1u, abort_flag)) { ok = false; site = 37; break; }
+            const TMeta mt = meta[it % kTMetaRing];
             if (mt.n == 0) break;
-            const int sb = it & 1u;
-            if (mt.first) { m = -INFINITY; l = 0.f; }
-            if (!mbar_wait(s_full(sb), (it >> 1) & 1u, abort_flag)) { ok = false; site = 38; break; }
-            tc_fence_after_sync();
-            uint32_t raw[2][32];
-            tmem_ld32(lane_base + sb * kTile, raw[0]);
-            tmem_ld32(lane_base + sb * kTile + 32, raw[1]);
-            tmem_wait_ld();
-            tc_fence_before_sync();
-            mbar_arrive(s_free(sb));
-            float mx = -INFINITY;
-            #pragma unroll
-            for (int h = 0; h < 2; ++h)
-                #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float v = __uint_as_float(raw[h][e]) * p.scale_log2e;
-                    raw[h][e] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
+            const bool warp_live = (warp & 3) * 4 < mt.n;        // this warp holds rows of a sharing sibling
+            const bool mine = (int)(it & 1u) == g;
+            if (g == 0 && mt.idx == 0) {
+                // ---- a segment starts: group A moves its queries from the staging buffer to TMEM
+                //      (row r of both 64-dim halves -> 64 columns of packed bf16 in lane r)
+                if (!mbar_wait(q_full(mt.qsel), (qsegs >> 1) & 1u, abort_flag)) { ok = false; site = 44; break; }
+                if (qsegs > 0) {
+                    if (!mbar_wait(qt_free, (qsegs - 1) & 1u, abort_flag)) { ok = false; site = 45; break; }
+                    tc_fence_after_sync();
                 }
-            const float m_new = fmaxf(m, mx);
-            const float alpha = fast_exp2(m - m_new);            // 0 on a segment's first tile
-            const bool moved = (m_new != m) && !mt.first;
-            // P.V of the previous tile must be complete: it reads the P tile written below, and a
-            // rescale must see all of O
-            if (it > 0) {
-                if (!mbar_wait(pv_done, (it - 1) & 1u, abort_flag)) { ok = false; site = 39; break; }
-                tc_fence_after_sync();
-            }
-            if (__any_sync(0xffffffffu, moved)) {
-                const float a = moved ? alpha : 1.f;
+                const uint8_t* qsrc = smem + TSmem::kQOff + mt.qsel * kTQBytes + row * 128;
                 #pragma unroll
-                for (int cblk = 0; cblk < 4; ++cblk) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_base + kTmemO + cblk * 32, o);
-                    tmem_wait_ld();
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t qw[32];
                     #pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
-                    tmem_st32(lane_base + kTmemO + cblk * 32, o);
+                    for (int ch = 0; ch < 8; ++ch) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (row < kTQRows) v = *reinterpret_cast<const uint4*>(qsrc + h * kTQHalfBytes + ((ch ^ sw) << 4));
+                        qw[4 * ch] = v.x; qw[4 * ch + 1] = v.y; qw[4 * ch + 2] = v.z; qw[4 * ch + 3] = v.w;
+                    }
+                    tmem_st32(lane_base + kTmemQ + h * 32, qw);
                 }
                 tmem_wait_st();
-            }
-            m = m_new;
-            float sum = 0.f;
-            #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {                     // 8 tokens = one 16-byte chunk of the P row
-                uint32_t w[4];
-                #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int t0 = ch * 8 + 2 * e;
-                    const float p0 = fast_exp2(__uint_as_float(raw[t0 >> 5][t0 & 31]) - m);
-                    const float p1 = fast_exp2(__uint_as_float(raw[(t0 + 1) >> 5][(t0 + 1) & 31]) - m);
-                    sum += p0 + p1;
-                    w[e] = pack_bf16(p0, p1);
-                }
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                             ::"r"(p_row + (uint32_t)((ch ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-            }
-            l = fmaf(l, alpha, sum);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            tc_fence_before_sync();
-            mbar_arrive(p_full);
-
-            if (mt.last) {
-                // ---- the segment's result: one normalised partial per sibling
-                if (!mbar_wait(pv_done, it & 1u, abort_flag)) { ok = false; site = 40; break; }
-                tc_fence_after_sync();
-                const float inv = 1.f / l;
-                const bool live = j < mt.n;
-                float* dst = c.pre_o + ((int64_t)(mt.row + j) * kGroup + head) * kD;
-                #pragma unroll
-                for (int cblk = 0; cblk < 4; ++cblk) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_base + kTmemO + cblk * 32, o);
-                    tmem_wait_ld();
-                    if (live) {
-                        #pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            *reinterpret_cast<float4*>(dst + cblk * 32 + e) =
-                                make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
-                                            __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-                    }
-                }
-                if (live) c.pre_lse[(int64_t)(mt.row + j) * kGroup + head] = m + log2f(l);
                 tc_fence_before_sync();
+                mbar_arrive(q_empty(mt.qsel));                   // the staging buffer may be refilled
+                mbar_arrive(qt_ready);
+                ++qsegs;
+            }
+            if (mine) {
+                const bool first = mt.idx < 2;                   // this group's first tile of the segment
+                if (!mbar_wait(s_full(g), k & 1u, abort_flag)) { ok = false; site = 38; break; }
+                tc_fence_after_sync();
+                uint32_t pk[32];                                 // the row's 64 probabilities, bf16 pairs
+                float sum = 0.f, alpha = 1.f, m_use = m_ref;
+                bool need = false;
+                if (warp_live) {
+                    uint32_t raw[2][32];
+                    tmem_ld32(lane_base + kTmemS + g * kTile, raw[0]);
+                    tmem_ld32(lane_base + kTmemS + g * kTile + 32, raw[1]);
+                    tmem_wait_ld();
+                    tc_fence_before_sync();
+                    mbar_arrive(s_free(g));
+                    // extreme raw score of the tile (two chains); the scale may be negative
+                    float e0 = __uint_as_float(raw[0][0]), e1 = __uint_as_float(raw[1][0]);
+                    if (!sc_neg) {
+                        #pragma unroll
+                        for (int e = 1; e < 31; e += 2) {
+                            asm("max.f32 %0, %0, %1, %2;" : "+f"(e0) : "f"(__uint_as_float(raw[0][e])), "f"(__uint_as_float(raw[0][e + 1])));
+                            asm("max.f32 %0, %0, %1, %2;" : "+f"(e1) : "f"(__uint_as_float(raw[1][e])), "f"(__uint_as_float(raw[1][e + 1])));
+                        }
+                        asm("max.f32 %0, %0, %1, %2;" : "+f"(e0) : "f"(__uint_as_float(raw[0][31])), "f"(__uint_as_float(raw[1][31])));
+                        e0 = fmaxf(e0, e1);
+                    } else {
+                        #pragma unroll
+                        for (int e = 1; e < 31; e += 2) {
+                            asm("min.f32 %0, %0, %1, %2;" : "+f"(e0) : "f"(__uint_as_float(raw[0][e])), "f"(__uint_as_float(raw[0][e + 1])));
+                            asm("min.f32 %0, %0, %1, %2;" : "+f"(e1) : "f"(__uint_as_float(raw[1][e])), "f"(__uint_as_float(raw[1][e + 1])));
+                        }
+                        asm("min.f32 %0, %0, %1, %2;" : "+f"(e0) : "f"(__uint_as_float(raw[0][31])), "f"(__uint_as_float(raw[1][31])));
+                        e0 = fminf(e0, e1);
+                    }
+                    const float mx = e0 * sc;
+                    need = !first && (mx > m_ref + kSlack);
+                    m_use = (first || need) ? mx : m_ref;
+                    if (need) alpha = fast_exp2(m_ref - mx);
+                    const float neg_m = -m_use;
+                    float sum1 = 0.f;
+                    #pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int t0 = 2 * e;
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(raw[t0 >> 5][t0 & 31]), sc, neg_m));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(raw[(t0 + 1) >> 5][(t0 + 1) & 31]), sc, neg_m));
+                        sum += p0; sum1 += p1;
+                        pk[e] = pack_bf16(p0, p1);
+                    }
+                    sum += sum1;
+                } else {
+                    tc_fence_before_sync();
+                    mbar_arrive(s_free(g));
+                }
+                // this group's previous P.V must be complete before its P tile is overwritten and
+                // before a rescale touches O; the probabilities above were computed while it ran
+                if (k > 0) {
+                    if (!mbar_wait(pv_done(g), (k - 1) & 1u, abort_flag)) { ok = false; site = 39; break; }
+                    tc_fence_after_sync();
+                }
+                if (warp_live) {
+                    if (__any_sync(0xffffffffu, need)) {
+                        #pragma unroll
+                        for (int cblk = 0; cblk < 4; ++cblk) {
+                            uint32_t o[32];
+                            tmem_ld32(o_mine + cblk * 32, o);
+                            tmem_wait_ld();
+                            #pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(o_mine + cblk * 32, o);
+                        }
+                        tmem_wait_st();
+                    }
+                    l = first ? sum : fmaf(l, alpha, sum);
+                    m_ref = m_use;
+                    tmem_st32(lane_base + kTmemP + g * 32, pk);  // the row's 64 probabilities, the A operand of P.V
+                    tmem_wait_st();
+                }
+                tc_fence_before_sync();
+                mbar_arrive(p_full(g));
+                ++k;
+            }
+
+            if (mt.idx == mt.cnt - 1) {
+                // ---- the segment ends with this tile: both groups meet, merge their two states of
+                //      every row and write one normalised partial per sibling (half the columns each)
+                const bool had = mine || mt.cnt >= 2;            // this group took a tile of the segment
+                if (had) {
+                    if (!mbar_wait(pv_done(g), (k - 1) & 1u, abort_flag)) { ok = false; site = 40; break; }
+                    tc_fence_after_sync();
+                }
+                xch[g * kTRows + row] = make_float2(had ? m_ref : -INFINITY, had ? l : 0.f);
+                mbar_arrive(xch_a);
+                if (!mbar_wait(xch_a, segs & 1u, abort_flag)) { ok = false; site = 41; break; }
+                if (warp_live) {
+                    const float2 other = xch[(g ^ 1) * kTRows + row];
+                    const bool had2 = other.y > 0.f;
+                    const float m1 = had ? m_ref : -INFINITY, l1 = had ? l : 0.f;
+                    const float M = fmaxf(m1, other.x);
+                    const float w1 = had ? fast_exp2(m1 - M) : 0.f, w2 = had2 ? fast_exp2(other.x - M) : 0.f;
+                    const float L = l1 * w1 + other.y * w2;
+                    const float inv = 1.f / L;
+                    const float f1 = w1 * inv, f2 = w2 * inv;
+                    const bool live = j < mt.n;
+                    float* dst = c.pre_o + ((int64_t)(mt.row + j) * kGroup + head) * kD + g * 64;
+                    #pragma unroll
+                    for (int cblk = 0; cblk < 2; ++cblk) {
+                        uint32_t oa[32], ob[32];
+                        if (had) tmem_ld32(o_mine + g * 64 + cblk * 32, oa);
+                        if (had2) tmem_ld32(o_other + g * 64 + cblk * 32, ob);
+                        tmem_wait_ld();
+                        if (live) {
+                            #pragma unroll
+                            for (int e = 0; e < 32; e += 4) {
+                                float4 v;
+                                float* vp = reinterpret_cast<float*>(&v);
+                                #pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const float a = had ? __uint_as_float(oa[e + q]) * f1 : 0.f;
+                                    vp[q] = had2 ? fmaf(__uint_as_float(ob[e + q]), f2, a) : a;
+                                }
+                                *reinterpret_cast<float4*>(dst + cblk * 32 + e) = v;
+                            }
+                        }
+                    }
+                    if (live && g == 0) c.pre_lse[(int64_t)(mt.row + j) * kGroup + head] = M + log2f(L);
+                }
+                // nobody's next P.V may overwrite an accumulator the other group is still reading
+                tc_fence_before_sync();
+                mbar_arrive(xch_b);
+                if (!mbar_wait(xch_b, segs & 1u, abort_flag)) { ok = false; site = 42; break; }
+                ++segs;
             }
         }
         if (!ok && lane == 0) wait_failed(p, abort_flag, site);

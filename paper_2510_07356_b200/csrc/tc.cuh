@@ -59,6 +59,18 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// D[tmem] (+)= A[tmem] . B[smem].  A occupies lanes 0..127 (row i = lane i) and, for 16-bit
+// types, 8 consecutive 32-bit columns per K = 16 step: column c holds elements 2c (low half)
+// and 2c + 1.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 // The mbarrier receives one arrival when every MMA this thread issued before has completed
 // (their shared-memory reads included).
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
