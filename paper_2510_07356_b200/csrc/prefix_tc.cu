@@ -194,13 +194,18 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
             if (!ok) return;
             const uint32_t vdst = smem_base + TSmem::kVOff + vs * kTTileBytes;
             mbar_arrive_expect_tx(full_v(vs), kTTileBytes);
-            #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (q < npages) {
-                    const int32_t prow = (m.pages[q] * kHkv + m.g) * P;
-                    tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(vs));
-                    tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(vs));
-                }
+            if (npages == 1) {
+                // page = tile: one box {64, 64, 2} lands as [half][row][128 B], the operand layout
+                tma_load_3d(vdst, &map_v, 0, (m.pages[0] * kHkv + m.g) * P, 0, full_v(vs));
+            } else {
+                #pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (q < npages) {
+                        const int32_t prow = (m.pages[q] * kHkv + m.g) * P;
+                        tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(vs));
+                        tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(vs));
+                    }
+            }
             ++vt;
         };
         int32_t r = blockIdx.x;
@@ -267,13 +272,17 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                             mbar_arrive(meta_full(it % kTMetaRing));
                             const uint32_t kdst = smem_base + ks * kTTileBytes;
                             mbar_arrive_expect_tx(full_k(ks), kTTileBytes);
-                            #pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                if (q < npages) {
-                                    const int32_t prow = (pages[q] * kHkv + g) * P;
-                                    tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
-                                    tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
-                                }
+                            if (npages == 1) {
+                                tma_load_3d(kdst, &map_k, 0, (pages[0] * kHkv + g) * P, 0, full_k(ks));
+                            } else {
+                                #pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    if (q < npages) {
+                                        const int32_t prow = (pages[q] * kHkv + g) * P;
+                                        tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
+                                        tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
+                                    }
+                            }
                             if (it >= (uint32_t)kTVLag) issue_v(it - kTVLag);
                         }
                     }
@@ -287,8 +296,13 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
         if (lane == 0) {
             while (ok && vt < it) issue_v(vt);                 // the last tiles' V
             if (ok) {
-                meta[it % kTMetaRing].n = 0;                   // no more work
-                mbar_arrive(meta_full(it % kTMetaRing));
+                const int ks = it % kTKStages;
+                ok = mbar_wait(empty_k(ks), ((it / kTKStages) & 1u) ^ 1u, abort_flag);
+                if (ok) {
+                    meta[it % kTMetaRing].n = 0;               // no more work
+                    mbar_arrive(meta_full(it % kTMetaRing));
+                    mbar_arrive(full_k(ks));                   // the Q.K^T warp reads records through the K barriers
+                }
             }
             if (!ok) {
                 wait_failed(p, abort_flag, 31);
@@ -301,20 +315,23 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
             }
         }
     } else if (warp == kTMmaWarp) {
-        // =========================================================== Q.K^T warp (one thread issues)
-        if (lane == 0) {
+        // =========================================================== Q.K^T warp (one lane issues)
+        // The whole warp runs the loop so that addresses and descriptors stay warp-uniform; the
+        // MMAs and commits are issued by lane 0.  The tile's record was written before its K
+        // barrier was armed, so waiting for K makes it visible; the end marker arrives the same way.
+        {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kTRows, kTile, false, false);
             bool ok = true;
             int site = 0;
             uint32_t segs = 0;
             for (uint32_t it = 0; ok; ++it) {
                 const int g = it & 1u;
-                if (!mbar_wait(meta_full(it % kTMetaRing), (it / kTMetaRing) & 1u, abort_flag)) { ok = false; site = 32; break; }
-                const TMeta mt = meta[it % kTMetaRing];
-                if (mt.n == 0) break;
                 const int ks = it % kTKStages;
                 if (!mbar_wait(full_k(ks), (it / kTKStages) & 1u, abort_flag)) { ok = false; site = 43; break; }
-                if (mt.idx == 0) {                            // a segment starts: its queries must be in TMEM
+                const TMeta* mt = &meta[it % kTMetaRing];
+                const int32_t idx = mt->idx, cnt = mt->cnt;
+                if (mt->n == 0) break;
+                if (idx == 0) {                               // a segment starts: its queries must be in TMEM
                     if (!mbar_wait(qt_ready, segs & 1u, abort_flag)) { ok = false; site = 33; break; }
                     ++segs;
                 }
@@ -322,17 +339,20 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                 if (!mbar_wait(s_free(g), ((it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; site = 34; break; }
                 tc_fence_after_sync();
                 const uint32_t k_addr = smem_base + ks * kTTileBytes;
-                #pragma unroll
-                for (int k16 = 0; k16 < 8; ++k16) {
-                    const uint32_t koff = (uint32_t)(k16 & 3) * 32u;
-                    const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
-                    umma_ts(tmem_base + kTmemS + g * kTile, tmem_base + kTmemQ + k16 * 8, b, idesc_qk, k16 > 0);
+                if (lane == 0) {
+                    #pragma unroll
+                    for (int k16 = 0; k16 < 8; ++k16) {
+                        const uint32_t koff = (uint32_t)(k16 & 3) * 32u;
+                        const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
+                        umma_ts(tmem_base + kTmemS + g * kTile, tmem_base + kTmemQ + k16 * 8, b, idesc_qk, k16 > 0);
+                    }
+                    umma_commit(s_full(g));
+                    umma_commit(empty_k(ks));                               // that K stage may be overwritten
+                    if (idx == cnt - 1) umma_commit(qt_free);              // the segment's last read of its queries
                 }
-                umma_commit(s_full(g));
-                umma_commit(empty_k(ks));                                   // that K stage may be overwritten
-                if (mt.idx == mt.cnt - 1) umma_commit(qt_free);            // the segment's last read of its queries
+                __syncwarp();
             }
-            if (!ok) wait_failed(p, abort_flag, site);
+            if (!ok && lane == 0) wait_failed(p, abort_flag, site);
         }
         __syncwarp();
     } else if (warp == kTPvWarp) {
@@ -583,12 +603,12 @@ EncodeTiledFn encode_fn() {
 // Rows of 128 bf16 seen as {64 elements, rows, 2 halves}; a box is `box_rows` rows of ONE half
 // and lands in shared memory as [row][128 B] with the 128-byte swizzle: one slab of a K-major
 // (or, read along the rows, MN-major) tcgen05 operand.
-bool make_half_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows) {
+bool make_half_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, uint32_t box_halves = 1) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {64, rows, 2};
     const cuuint64_t strides[2] = {256, 128};
-    const cuuint32_t box[3] = {64, box_rows, 1};
+    const cuuint32_t box[3] = {64, box_rows, box_halves};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -600,8 +620,10 @@ bool make_half_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32
 cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
     const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
-    if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.page_size) ||
-        !make_half_row_map(&mv, p.v_pages, pool_rows, p.page_size) ||
+    // a 64-token page is a whole tile: both halves come with one copy ([half][row][128 B])
+    const uint32_t halves = p.page_size == kTile ? 2 : 1;
+    if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.page_size, halves) ||
+        !make_half_row_map(&mv, p.v_pages, pool_rows, p.page_size, halves) ||
         !make_half_row_map(&mq, p.q, (uint64_t)p.batch * kHq, kGroup))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TSmem::kBytes);
