@@ -3,6 +3,10 @@ C ABI on seeded synthetic long-trace workloads.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
+NAME is one of synth.SPECS (plain decode step; the default is the 64 x 16,384 configuration) or of
+synth.CASCADE_SPECS (shared-prefix step: `value` counts the shared pages once, `logical_gbs` as if
+every sequence had read its whole context, `roofline` is the prefix-pass kernel).
+
 One JSON line on stdout (rank 0).  `value` is the algorithmic bytes of the step (K and V of
 every cached token, q/out/lse, used table entries) divided by the device time of the whole
 step with all inputs resident in HBM; `e2e` is the same through the host-buffer entry point
@@ -54,6 +58,7 @@ def parse_args():
     ap.add_argument("--loop-steps", type=int, default=16, help="append+attention steps replayed from a CUDA graph")
     ap.add_argument("--fuse-combine", type=int, default=-1)
     ap.add_argument("--claim-ahead", type=int, default=-1)
+    ap.add_argument("--prefix-kernel", type=int, default=0, help="cascade workloads: 0 tcgen05 prefix pass, 1 mma.sync")
     return ap.parse_args()
 
 
@@ -206,7 +211,12 @@ def run_reference(args):
     import numpy as np
     import synth
     # the sample is built from the workload's lengths without building its full pools
-    spec = synth.SPECS[args.workload]
+    if args.workload in synth.CASCADE_SPECS:     # the oracle reads every sequence's whole context itself
+        lens_list = [sh + o for sh, owns in synth.cascade_groups(args.workload) for o in owns]
+        spec = synth.tiny_spec(args.workload, lens_list, synth.CASCADE_SPECS[args.workload][4],
+                               synth.CASCADE_SPECS[args.workload][5])
+    else:
+        spec = synth.SPECS[args.workload]
     lens = synth.make_lengths(spec)
     cores = host_cores()
     # bounded sample: sequences in a seeded order, sized by a one-group calibration
@@ -246,10 +256,131 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_cascade(args):
+    """Shared-prefix (cascade) decode step on a named cascade workload, 1 GPU or replicas."""
+    import torch
+    import torch.distributed as dist
+    import synth
+    import paper_2510_07356_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    cw = synth.make_named_cascade(args.workload, dev)
+    w, spec = cw.w, cw.w.spec
+    attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
+    attn.set_option(P.CONCUR_OPT_PREFIX_KERNEL, args.prefix_kernel)
+    out = torch.empty_like(w.q)
+    lse = torch.empty((spec.batch, spec.num_q_heads), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    G = len(cw.prefix_lens_host)
+
+    def step():
+        P.concur_decode_attn_cascade(attn.handle, w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens,
+                                     cw.group_start, cw.prefix_lens, w.scale, out, lse, spec.batch, G,
+                                     w.num_pages, w.block_table.shape[1], stream.cuda_stream)
+
+    def plain_step():
+        attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale, out=out, lse=lse)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    K = args.steps
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    assert attn.status() == 0, "device-side flags set during warm-up"
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K + 2)]
+    for row in ev:
+        for e in row:
+            e.record(stream)
+    barrier()
+    t_mark0 = time.time()
+    ev[K][0].record(stream)
+    for _ in range(K):
+        step()
+    ev[K][1].record(stream)
+    barrier()
+    ms_per_step = ev[K][0].elapsed_time(ev[K][1]) / K
+    for i in range(K):                       # the same steps with events around the prefix-pass kernel
+        attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, ev[i][0].cuda_event)
+        attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, ev[i][1].cuda_event)
+        step()
+    barrier()
+    t_mark1 = time.time()
+    clocks = sampler.stop(t_mark0, t_mark1) if rank == 0 else None
+    attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, 0)
+    attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, 0)
+    pre_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
+    ev[K + 1][0].record(stream)              # the plain step on the same tables, for comparison
+    for _ in range(K):
+        plain_step()
+    ev[K + 1][1].record(stream)
+    barrier()
+    plain_ms = ev[K + 1][0].elapsed_time(ev[K + 1][1]) / K
+    ms_per_step, pre_ms_avg, plain_ms = over_ranks([ms_per_step, sum(pre_ms) / K, plain_ms], "max", dev)
+    shared_b, logical_b, pre_b = cw.shared_bytes(), cw.logical_bytes(), synth.cascade_prefix_bytes(cw)
+    job_shared, job_logical, job_tokens = over_ranks([shared_b, logical_b, w.kv_tokens], "sum", dev)
+    flags = attn.status()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peak()
+    value = job_shared / (ms_per_step * 1e-3) / 1e9
+    achieved = pre_b / (pre_ms_avg * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "groups": G, "kv_tokens_logical": w.kv_tokens,
+                   "page_size": spec.page_size, "heads": "64q/8kv", "head_dim": 128,
+                   "algorithmic_bytes": shared_b, "logical_bytes": logical_b, "prefix_pass_bytes": pre_b,
+                   "l2": "inputs larger than L2", "entry": "concur_decode_attn_cascade",
+                   "prefix_kernel": "tcgen05" if args.prefix_kernel == 0 else "mma.sync",
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+        "kv_tokens_per_s": job_tokens / (ms_per_step * 1e-3),
+        "logical_gbs": job_logical / (ms_per_step * 1e-3) / 1e9,
+        "plain_step_ms": plain_ms, "speedup_over_plain_step": plain_ms / ms_per_step,
+        "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
+        "frac_of_measured_copy": value / world / peak,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "prefix pass", "ms": pre_ms_avg,
+                     "ms_min": min(pre_ms)},
+        "e2e": None, "gpu_launches": 4 * K, "clocks": clocks, "device_flags": flags,
+    }
+    if not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload.startswith("casc"):
+        run_cascade(args)
         return
 
     import torch

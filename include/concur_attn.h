@@ -70,7 +70,8 @@ typedef enum {
 #define CONCUR_OPT_MIN_RANGE_TILES 5/* heuristic's smallest range, in 64-token tiles; 0 = default (2)   */
 #define CONCUR_OPT_EVENT_BEFORE_PARTIAL 6 /* a cudaEvent_t (as an integer) recorded on the call's stream
                                              just before the partial kernel; 0 = none.  For timing
-                                             that kernel alone; the event stays the caller's.          */
+                                             that kernel alone; the event stays the caller's.  In the
+                                             cascade step the two events bracket the prefix-pass kernel. */
 #define CONCUR_OPT_EVENT_AFTER_PARTIAL  7 /* likewise, just after the partial kernel                    */
 #define CONCUR_OPT_FUSE_COMBINE 8   /* tensor-core kernel: 1 (default) = the CTA that finishes a unit's last
                                        partial merges the unit in-kernel; 0 = separate combine kernel   */

@@ -303,8 +303,10 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (launch_plan_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    if (h->ev_before && cudaEventRecord(h->ev_before, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if ((h->prefix_kernel == 1 ? launch_prefix_mma(p, c, stream) : launch_prefix_tc(p, c, stream)) != cudaSuccess)
         return CONCUR_ERR_CUDA;
+    if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream);
     if (e != cudaSuccess) return CONCUR_ERR_CUDA;
     if (launch_combine_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;

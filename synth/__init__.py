@@ -318,3 +318,39 @@ def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0
     pl = np.asarray(pre, dtype=np.int32)
     return CascadeWorkload(w=w, group_start=torch.from_numpy(gs).to(device), prefix_lens=torch.from_numpy(pl).to(device),
                            group_start_host=gs, prefix_lens_host=pl)
+
+
+# Shared-prefix decode workloads: (tasks, samples per task, shared prompt tokens, range of each
+# sample's own tokens, page size, seed).  Shaped like the sampling of the paper's pipeline: one
+# fixed prompt per task, 5 samples per task in synthesis and 10 in evaluation, traces of a few
+# thousand tokens; the third is a long-prompt stress case for the prefix pass.
+CASCADE_SPECS = {
+    "casc_24x10_pre2048_p64": (24, 10, 2048, (256, 8192), 64, 73571),
+    "casc_32x5_pre2048_p64": (32, 5, 2048, (256, 8192), 64, 73572),
+    "casc_16x10_pre16384_p64": (16, 10, 16384, (1, 256), 64, 73573),
+}
+
+
+def cascade_groups(name: str):
+    """[(shared tokens, [own tokens per sample])] of a named cascade workload."""
+    tasks, samples, shared, (a, b), page_size, seed = CASCADE_SPECS[name]
+    r = _rng(seed, 7)
+    return [(shared, r.integers(a, b + 1, size=samples).tolist()) for _ in range(tasks)]
+
+
+def make_named_cascade(name: str, device="cpu") -> CascadeWorkload:
+    page_size, seed = CASCADE_SPECS[name][4], CASCADE_SPECS[name][5]
+    return make_cascade_workload(name, cascade_groups(name), page_size, seed, device)
+
+
+def cascade_prefix_bytes(cw: CascadeWorkload) -> int:
+    """Bytes the prefix pass must read: K and V of every group's shared whole 64-token tiles
+    (counted once per group) plus the sharing siblings' query rows per KV head."""
+    s = cw.w.spec
+    per_token = 2 * s.num_kv_heads * s.head_dim * 2
+    total = 0
+    for i, pre in enumerate(cw.prefix_lens_host):
+        n = int(cw.group_start_host[i + 1] - cw.group_start_host[i])
+        if n >= 2:
+            total += (int(pre) // 64) * 64 * per_token + n * s.num_q_heads * s.head_dim * 2
+    return total
