@@ -156,7 +156,7 @@ def host_cores():
 
 
 def cpu_baseline(w, target_seconds):
-    """Oracle throughput on a bounded sample of the workload's sequences (all 64 heads each)."""
+    """Oracle throughput on a bounded sample of the workload's sequences (all query heads each)."""
     import numpy as np
     import synth
     cores = host_cores()
@@ -181,7 +181,7 @@ def cpu_baseline(w, target_seconds):
     dt = oracle_sample_throughput(sub, list(range(len(seqs))), cores)
     nbytes = sub.algorithmic_bytes()
     return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{len(seqs)} of {w.spec.batch} sequences ({tok} of {w.kv_tokens} KV tokens), all 64 heads, "
+            "sample": f"{len(seqs)} of {w.spec.batch} sequences ({tok} of {w.kv_tokens} KV tokens), all {w.spec.num_q_heads} query heads, "
                       f"{dt:.1f} s wall", "kv_tokens_per_s": tok / dt}
 
 
@@ -222,7 +222,7 @@ def run_reference(args):
     # bounded sample: sequences in a seeded order, sized by a one-group calibration
     order = np.random.default_rng(7).permutation(spec.batch).tolist()
     probe = synth.make_workload(synth.tiny_spec("probe", (int(lens[order[0]]),), spec.page_size, spec.seed,
-                                                q_std=spec.q_std), "cpu")
+                                                q_std=spec.q_std, num_q_heads=spec.num_q_heads), "cpu")
     import oracle
     oracle.build()
     t0 = time.perf_counter()
@@ -238,14 +238,14 @@ def run_reference(args):
             break
     sample = synth.make_workload(
         synth.tiny_spec("sample", [int(lens[b]) for b in seqs], spec.page_size, spec.seed, q_std=spec.q_std,
-                        k_outlier_prob=spec.k_outlier_prob), "cpu")
+                        k_outlier_prob=spec.k_outlier_prob, num_q_heads=spec.num_q_heads), "cpu")
     for _ in range(args.warmup):
         oracle_sample_throughput(sample, list(range(len(seqs))), cores)
     t = [oracle_sample_throughput(sample, list(range(len(seqs))), cores) for _ in range(args.steps)]
     dt = sum(t) / len(t)
     nbytes = sample.algorithmic_bytes()
     value = nbytes / dt / 1e9
-    desc = (f"{len(seqs)} of {spec.batch} sequences ({tok} of {int(lens.sum())} KV tokens), all 64 heads, per step")
+    desc = (f"{len(seqs)} of {spec.batch} sequences ({tok} of {int(lens.sum())} KV tokens), all {spec.num_q_heads} query heads, per step")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -402,7 +402,8 @@ def main():
     # every rank decodes its own batch of the same shape (replicas, no data-path collective)
     spec = rank_spec(synth.SPECS[args.workload], rank, world)
     w = synth.make_workload(spec, dev, spare_tokens=args.loop_steps)
-    attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
+    attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local,
+                             num_q_heads=spec.num_q_heads)
     attn.set_option(P.CONCUR_OPT_KERNEL, args.kernel)
     attn.set_option(P.CONCUR_OPT_RANGES_PER_CTA, args.ranges_per_cta)
     attn.set_option(P.CONCUR_OPT_MIN_RANGE_TILES, args.min_range_tiles)
@@ -559,7 +560,7 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": spec.name, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
-                   "heads": "64q/8kv", "head_dim": 128, "algorithmic_bytes": nbytes,
+                   "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128, "algorithmic_bytes": nbytes,
                    "l2": "flushed between steps" if flush_needed else "inputs larger than L2",
                    "kernel": "mma" if args.kernel == 0 else "scalar", "ranges": R, "tiles": W,
                    "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},

@@ -2,7 +2,7 @@
  * concur_attn -- paged-KV grouped-query decode attention for NVIDIA B200 (sm_100a).
  *
  * One call computes one decode step of one layer:  for every sequence b of the batch
- * and every query head h (KV head g = h / (Hq/Hkv)), over the n = seq_lens[b] tokens
+ * and every query head h (KV head g = h / (Hq/Hkv), Hq/Hkv = 1 .. 8), over the n = seq_lens[b] tokens
  * cached for that sequence,
  *
  *     s_j   = scale * <q[b][h], K[token j of b][g]>
@@ -84,8 +84,8 @@ typedef enum {
 typedef struct concur_attn concur_attn_t;   /* opaque; owns its workspace and nothing else */
 
 typedef struct {
-    int32_t num_q_heads;        /* Hq; supported: 64                                            */
-    int32_t num_kv_heads;       /* Hkv; supported: 8 (group size Hq/Hkv = 8)                    */
+    int32_t num_q_heads;        /* Hq; supported: 8, 16, ... 64 (group size Hq/Hkv = 1 .. 8), e.g. 64 or 40 */
+    int32_t num_kv_heads;       /* Hkv; supported: 8                                            */
     int32_t head_dim;           /* D; supported: 128                                            */
     int32_t page_size;          /* P; supported: 16, 32, 64 tokens                              */
     int32_t max_batch;          /* largest `batch` any call will pass (1 .. 65536)              */
@@ -242,7 +242,8 @@ int concur_attn_last_plan(concur_attn_t* handle, void* cuda_stream, int32_t* num
  * array inside the library's device image -- about 4.3 MB that every GPU which loads the
  * library holds until the process exits -- and there is no handle at all.
  *
- * Arguments and layouts are those of concur_decode_attn, plus `page_size` (16, 32 or 64);
+ * Arguments and layouts are those of concur_decode_attn for 64 query heads and 8 KV heads, plus
+ * `page_size` (16, 32 or 64);
  * the work is enqueued on `cuda_stream` of the CURRENT device and the call returns without
  * synchronising.  It performs no cudaMalloc / cudaFree and calls no allocating library
  * routine.  Limits: batch <= CONCUR_STATIC_MAX_BATCH (more: CONCUR_ERR_TOO_LARGE, nothing

@@ -38,7 +38,8 @@ int check_config(const concur_attn_config_t* c) {
     if (c->reserved != 0 || c->device < 0) return CONCUR_ERR_INVALID_ARG;
     if (c->max_batch < 1 || c->max_batch > kMaxBatchLimit) return CONCUR_ERR_INVALID_ARG;
     if (c->max_pages_per_seq < 1) return CONCUR_ERR_INVALID_ARG;
-    if (c->num_q_heads != kHq || c->num_kv_heads != kHkv || c->head_dim != kD) return CONCUR_ERR_UNSUPPORTED;
+    if (c->num_kv_heads != kHkv || c->head_dim != kD) return CONCUR_ERR_UNSUPPORTED;
+    if (c->num_q_heads < kHkv || c->num_q_heads > kHq || c->num_q_heads % kHkv != 0) return CONCUR_ERR_UNSUPPORTED;
     if (c->page_size != 16 && c->page_size != 32 && c->page_size != 64) return CONCUR_ERR_UNSUPPORTED;
     // the flat tile index space must fit int32
     const int64_t tiles_per_seq = ((int64_t)c->max_pages_per_seq * c->page_size + kTile - 1) / kTile;
@@ -148,6 +149,8 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.bt_stride = stride;
     p.page_size = h->cfg.page_size;
     p.page_shift = h->cfg.page_size == 16 ? 4 : (h->cfg.page_size == 32 ? 5 : 6);
+    p.hq = h->cfg.num_q_heads;
+    p.group = h->cfg.num_q_heads / kHkv;
     const int per_sm = h->kernel == 1 ? partial_scalar_ctas_per_sm() : 1;
     p.grid_ctas = h->grid_ctas > 0 ? h->grid_ctas : h->sm_count * per_sm;
     p.forced_ranges = h->forced_ranges;
@@ -332,11 +335,11 @@ int concur_decode_attn_host(concur_attn_t* h, const void* q, const void* k_pages
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok()) return CONCUR_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t q_bytes = (size_t)batch * kHq * kD * 2;
+    const size_t q_bytes = (size_t)batch * h->cfg.num_q_heads * kD * 2;
     const size_t pool_bytes = (size_t)num_pages * kHkv * h->cfg.page_size * kD * 2;
     const size_t bt_bytes = (size_t)batch * block_table_stride * 4;
     const size_t len_bytes = (size_t)batch * 4;
-    const size_t lse_bytes = (size_t)batch * kHq * 4;
+    const size_t lse_bytes = (size_t)batch * h->cfg.num_q_heads * 4;
     if ((rc = ensure(h->st_q, q_bytes)) || (rc = ensure(h->st_k, pool_bytes)) ||
         (rc = ensure(h->st_v, pool_bytes)) || (rc = ensure(h->st_bt, bt_bytes)) ||
         (rc = ensure(h->st_len, len_bytes)) || (rc = ensure(h->st_out, q_bytes)) ||

@@ -13,9 +13,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     const int b = blockIdx.x / kHkv, g = blockIdx.x % kHkv;
     const int d = threadIdx.x;
     const int32_t tiles_b = p.tiles_prefix[b + 1] - p.tiles_prefix[b];
-    const int64_t row0 = (int64_t)b * kHq + g * kGroup;
+    const int64_t row0 = (int64_t)b * p.hq + g * p.group;
     if (tiles_b == 0) {                       // no cached token: out = 0, lse = -inf
-        for (int h = 0; h < kGroup; ++h) {
+        for (int h = 0; h < p.group; ++h) {
             p.out[(row0 + h) * kD + d] = __float2bfloat16_rn(0.f);
             if (d == 0) p.lse[row0 + h] = -INFINITY;
         }
@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     // the unit's segment in range r is the range's first segment unless the range began
     // before the unit did (possible for r_lo only)
     const int32_t slot_lo = 2 * r_lo + (p.range_start[r_lo] < unit_start ? 1 : 0);
-    for (int h = 0; h < kGroup; ++h) {
+    for (int h = 0; h < p.group; ++h) {
         float M = p.part_lse[(int64_t)slot_lo * kGroup + h];
         for (int32_t r = r_lo + 1; r <= r_hi; ++r)
             M = fmaxf(M, p.part_lse[(int64_t)(2 * r) * kGroup + h]);
@@ -105,9 +105,10 @@ __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(Decode
             add(c.pre_lse + row * kGroup, c.pre_o + row * kGroup * kD);
         }
     }
-    const int64_t row0 = (int64_t)b * kHq + g * kGroup;
+    const int64_t row0 = (int64_t)b * p.hq + g * p.group;
     #pragma unroll
     for (int h = 0; h < kGroup; ++h) {
+        if (h >= p.group) break;
         const bool any = z[h] > 0.f;
         p.out[(row0 + h) * kD + d] = __float2bfloat16_rn(any ? acc[h] / z[h] : 0.f);
         if (d == 0) p.lse[row0 + h] = any ? (mx[h] + log2f(z[h])) * 0.6931471805599453f : -INFINITY;

@@ -10,7 +10,7 @@ namespace concur {
 
 constexpr int kHq = 64;          // query heads
 constexpr int kHkv = 8;          // KV heads
-constexpr int kGroup = 8;        // query heads per KV head
+constexpr int kGroup = 8;        // most query heads per KV head; width of every partial slot
 constexpr int kD = 128;          // head dimension
 constexpr int kTile = 64;        // tokens per KV tile: the unit the plan counts in
 constexpr int kRowBytes = kD * 2;
@@ -44,6 +44,8 @@ struct DecodeParams {
     int32_t bt_stride;
     int32_t page_size;
     int32_t page_shift;       // log2(page_size)
+    int32_t group;            // query heads per KV head (1..kGroup); heads g*group .. g*group+group-1 share KV head g
+    int32_t hq;               // query heads = kHkv * group
     // plan controls
     int32_t grid_ctas;        // CTAs the partial kernel is launched with
     int32_t forced_ranges;    // > 0: use exactly this many ranges (clamped to [1, min(W, max_ranges)])

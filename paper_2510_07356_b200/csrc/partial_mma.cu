@@ -123,6 +123,13 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (p.group < kGroup) {
+        // fewer than 8 heads per group: the query rows that no copy fills must at least be defined
+        for (int i = tid; i < kStages * (kQBytes / 16); i += kThreads)
+            reinterpret_cast<uint4*>(smem + (i / (kQBytes / 16)) * kStageBytes + 2 * kTileBytes)[i % (kQBytes / 16)] =
+                make_uint4(0, 0, 0, 0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     // everything above overlaps the plan kernel when launched as its programmatic dependent;
     // the plan's outputs are read only below this wait
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -207,10 +214,11 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                             const uint32_t kdst = smem_base + s * kStageBytes;
                             const uint32_t vdst = kdst + kTileBytes;
                             const bool with_q = (t == sg.tile0);
-                            mbar_arrive_expect_tx(full_k(s), npages * box_bytes + (with_q ? kQBytes : 0));
+                            const uint32_t q_bytes = (uint32_t)p.group * kRowBytes;
+                            mbar_arrive_expect_tx(full_k(s), npages * box_bytes + (with_q ? q_bytes : 0));
                             if (with_q)
-                                bulk_load(vdst + kTileBytes, p.q + ((int64_t)sg.b * kHq + sg.g * kGroup) * kD,
-                                          kQBytes, full_k(s));
+                                bulk_load(vdst + kTileBytes, p.q + ((int64_t)sg.b * p.hq + sg.g * p.group) * kD,
+                                          q_bytes, full_k(s));
                             const int32_t pages[4] = {page0, page1, page2, page3};
                             #pragma unroll
                             for (int i = 0; i < 4; ++i)
@@ -311,8 +319,9 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             }
             #pragma unroll
             for (int h = 0; h < kGroup; ++h) {
+                if (h >= p.group) break;
                 const float inv = 1.f / z[h];
-                const int64_t row = (int64_t)jb * kHq + jg * kGroup + h;
+                const int64_t row = (int64_t)jb * p.hq + jg * p.group + h;
                 uint2 packed;
                 packed.x = pack_bf16(acc[h].x * inv, acc[h].y * inv);
                 packed.y = pack_bf16(acc[h].z * inv, acc[h].w * inv);
@@ -499,9 +508,11 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 const float res = acc / L;
                 const float lse2 = M + log2f(L);
                 if (mt.slot < 0) {
-                    const int64_t row = (int64_t)mt.b * kHq + mt.g * kGroup + h;
-                    p.out[row * kD + d] = __float2bfloat16_rn(res);
-                    if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
+                    if (h < p.group) {
+                        const int64_t row = (int64_t)mt.b * p.hq + mt.g * p.group + h;
+                        p.out[row * kD + d] = __float2bfloat16_rn(res);
+                        if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
+                    }
                 } else {
                     const int64_t row = (int64_t)mt.slot * kGroup + h;
                     p.part_o[row * kD + d] = res;

@@ -60,10 +60,11 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
             float q[kGroup][8];
             {
                 const uint4* qp = reinterpret_cast<const uint4*>(
-                    p.q + ((int64_t)sg.b * kHq + sg.g * kGroup) * kD) + sub;
+                    p.q + ((int64_t)sg.b * p.hq + sg.g * p.group) * kD) + sub;
                 #pragma unroll
                 for (int h = 0; h < kGroup; ++h) {
-                    unpack8(__ldg(qp + h * (kD / 8)), q[h]);
+                    // heads beyond the group size compute on zeros and are never written out
+                    unpack8(h < p.group ? __ldg(qp + h * (kD / 8)) : make_uint4(0, 0, 0, 0), q[h]);
                     #pragma unroll
                     for (int e = 0; e < 8; ++e) q[h][e] *= p.scale_log2e;
                 }
@@ -175,9 +176,11 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
                 const float res = acc / L;
                 const float lse2 = M + log2f(L);
                 if (sg.slot < 0) {
-                    const int64_t row = (int64_t)sg.b * kHq + sg.g * kGroup + h;
-                    p.out[row * kD + d] = __float2bfloat16_rn(res);
-                    if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
+                    if (h < p.group) {
+                        const int64_t row = (int64_t)sg.b * p.hq + sg.g * p.group + h;
+                        p.out[row * kD + d] = __float2bfloat16_rn(res);
+                        if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
+                    }
                 } else {
                     const int64_t row = (int64_t)sg.slot * kGroup + h;
                     p.part_o[row * kD + d] = res;

@@ -41,10 +41,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
         while (empties) {
             const int e = base + warp * 32 + (__ffs(empties) - 1);
             empties &= empties - 1;
-            uint4* o = reinterpret_cast<uint4*>(p.out + (int64_t)e * kHq * kD);
-            for (int i = lane; i < kHq * kD / 8; i += 32) o[i] = make_uint4(0, 0, 0, 0);
-            p.lse[(int64_t)e * kHq + lane] = -INFINITY;
-            p.lse[(int64_t)e * kHq + 32 + lane] = -INFINITY;
+            uint4* o = reinterpret_cast<uint4*>(p.out + (int64_t)e * p.hq * kD);
+            for (int i = lane; i < p.hq * kD / 8; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+            for (int i = lane; i < p.hq; i += 32) p.lse[(int64_t)e * p.hq + i] = -INFINITY;
         }
         // inclusive scan over the block
         int32_t v = tiles;

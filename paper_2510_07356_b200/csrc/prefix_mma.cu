@@ -160,7 +160,7 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                                 mbar_arrive_expect_tx(q_full(qsel), n * kQTileBytes);
                                 const uint32_t qdst = smem_base + L::kQOff + qsel * NS * kQTileBytes;
                                 for (int j = 0; j < n; ++j)
-                                    tma_load_tile(qdst + j * kQTileBytes, &map_q, ((b0 + j) * kHq + g * kGroup), q_full(qsel));
+                                    tma_load_tile(qdst + j * kQTileBytes, &map_q, ((b0 + j) * p.hq + g * p.group), q_full(qsel));
                             }
                         }
                         if (ok) {
@@ -460,7 +460,7 @@ cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cud
     CUtensorMap mk, mv, mq;
     const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
     if (!make_row_map(&mk, p.k_pages, pool_rows, p.page_size) || !make_row_map(&mv, p.v_pages, pool_rows, p.page_size) ||
-        !make_row_map(&mq, p.q, (uint64_t)p.batch * kHq, kGroup))
+        !make_row_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup))
         return cudaErrorInvalidValue;
     return launch_ns<kMaxShare>(p, c, mk, mv, mq, stream);
 }

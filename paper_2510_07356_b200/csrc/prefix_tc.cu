@@ -258,7 +258,7 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                                 mbar_arrive_expect_tx(q_full(qsel), n * kGroup * kRowBytes);
                                 const uint32_t qdst = smem_base + TSmem::kQOff + qsel * kTQBytes;
                                 for (int j = 0; j < n; ++j) {
-                                    const int32_t qrow = (b0 + j) * kHq + g * kGroup;
+                                    const int32_t qrow = (b0 + j) * p.hq + g * p.group;
                                     tma_load_3d(qdst + j * 1024, &map_q, 0, qrow, 0, q_full(qsel));
                                     tma_load_3d(qdst + kTQHalfBytes + j * 1024, &map_q, 0, qrow, 1, q_full(qsel));
                                 }
@@ -624,7 +624,7 @@ cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cuda
     const uint32_t halves = p.page_size == kTile ? 2 : 1;
     if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.page_size, halves) ||
         !make_half_row_map(&mv, p.v_pages, pool_rows, p.page_size, halves) ||
-        !make_half_row_map(&mq, p.q, (uint64_t)p.batch * kHq, kGroup))
+        !make_half_row_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TSmem::kBytes);
     if (e != cudaSuccess) return e;

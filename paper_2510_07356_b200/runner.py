@@ -10,11 +10,12 @@ class DecodeAttention:
     """Owns one concur_attn handle.  `__call__` enqueues one decode-attention step on
     torch's current stream and returns (out bf16 [B][Hq][D], lse fp32 [B][Hq])."""
 
-    def __init__(self, page_size: int, max_batch: int, max_pages_per_seq: int, device: int = 0):
+    def __init__(self, page_size: int, max_batch: int, max_pages_per_seq: int, device: int = 0,
+                 num_q_heads: int = 64):
         if not torch.cuda.is_available():
             raise RuntimeError("concur_attn needs a CUDA device; there is no CPU path")
         self.device = torch.device("cuda", device)
-        self.cfg = B.make_config(page_size, max_batch, max_pages_per_seq, device)
+        self.cfg = B.make_config(page_size, max_batch, max_pages_per_seq, device, num_q_heads=num_q_heads)
         self.handle = B.concur_attn_create(self.cfg)
 
     def set_option(self, key: int, value: int):

@@ -58,6 +58,9 @@ SPECS = {
     "cfg3_b64_ctx16384_p64": Spec("cfg3_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563),
     # a quarter of cfg3 (same lengths, page size and values): small enough for profiler captures
     "cfg3q_b16_ctx16384_p64": Spec("cfg3q_b16_ctx16384_p64", 16, 64, ("const", 16384), q_std=0.5, seed=73563),
+    # config 3 with 40 query heads (group size 5): the geometry variant of the same workload
+    "cfg3h40_b64_ctx16384_p64": Spec("cfg3h40_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563,
+                                     num_q_heads=40),
     "cfg4_b256_logu2k_32k_p64": Spec("cfg4_b256_logu2k_32k_p64", 256, 64, ("loguniform", 2048, 32768), seed=73564),
     "cfg5_b32_skew128k_p64": Spec("cfg5_b32_skew128k_p64", 32, 64, ("skew", 131072, 256, 4096),
                                   k_outlier_prob=0.01, seed=73565),
@@ -264,7 +267,8 @@ class CascadeWorkload:
         return self.w.algorithmic_bytes() - saved
 
 
-def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0) -> CascadeWorkload:
+def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0,
+                          num_q_heads=NUM_Q_HEADS) -> CascadeWorkload:
     """groups: list of (shared_tokens, [own_tokens of each sibling]).  `shared_tokens` must be a
     multiple of the page size (only whole pages can be shared physically).  Sequence lengths are
     shared + own; siblings point at the same physical pages for the shared part; all pages are
@@ -277,7 +281,8 @@ def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0
         gstart.append(len(lens))
         pre.append(shared)
     lens = np.asarray(lens, dtype=np.int32)
-    spec = Spec(name, len(lens), P, ("list", [int(x) for x in lens]), seed=seed, q_std=q_std)
+    spec = Spec(name, len(lens), P, ("list", [int(x) for x in lens]), seed=seed, q_std=q_std,
+                num_q_heads=num_q_heads)
     # page allocation: shared pages once per group, then each sibling's own pages
     rows, total = [], 0
     for (shared, owns), b0 in zip(groups, gstart[:-1]):

@@ -39,7 +39,9 @@ def test_workspace_bytes_and_config_checks(P):
     assert n > 2 * 4096 * 8 * 128 * 4 and n % 256 == 0
     bigger = P.concur_attn_workspace_bytes(P.make_config(64, 4096, 512))
     assert bigger > n
-    assert P.concur_attn_workspace_bytes(P.make_config(64, 256, 512, num_q_heads=40)) == 0
+    assert P.concur_attn_workspace_bytes(P.make_config(64, 256, 512, num_q_heads=40)) == n      # group size 5
+    assert P.concur_attn_workspace_bytes(P.make_config(64, 256, 512, num_q_heads=44)) == 0      # not a multiple of 8
+    assert P.concur_attn_workspace_bytes(P.make_config(64, 256, 512, num_q_heads=72)) == 0
     assert P.concur_attn_workspace_bytes(P.make_config(48, 256, 512)) == 0
     assert P.concur_attn_workspace_bytes(P.make_config(64, 0, 512)) == 0
 
