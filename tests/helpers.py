@@ -29,16 +29,23 @@ def oracle_sequences(w, seqs=None, threads=None):
     seqs = list(range(w.spec.batch)) if seqs is None else list(seqs)
     qb = oracle._u16(w.q); kb = oracle._u16(w.k_pages); vb = oracle._u16(w.v_pages)
     tb = oracle._i32(w.block_table); lb = oracle._i32(w.seq_lens)
-
-    def one(b):
-        o, l = oracle.decode_attn(qb, kb, vb, tb, lb, w.scale, seqs=(b, b + 1))
-        return o[b], l[b]
-
-    with ThreadPoolExecutor(max_workers=threads or host_cores()) as ex:
-        res = list(ex.map(one, seqs))
-    if not res:
+    threads = threads or host_cores()
+    if not seqs:
         return np.zeros((0, w.spec.num_q_heads, w.spec.head_dim)), np.zeros((0, w.spec.num_q_heads))
-    return np.stack([r[0] for r in res]), np.stack([r[1] for r in res])
+    # a few chunks of sequences per thread; each call gets only its chunk's rows of q, of the
+    # table and of the lengths, so that its result arrays are chunk-sized (a call over the whole
+    # batch allocates batch-sized results, which for thousands of short sequences is gigabytes)
+    idx = np.asarray(seqs, dtype=np.int64)
+    nchunks = min(len(seqs), threads * 4)
+    chunks = [c for c in np.array_split(idx, nchunks) if len(c)]
+
+    def one(c):
+        return oracle.decode_attn(np.ascontiguousarray(qb[c]), kb, vb, np.ascontiguousarray(tb[c]),
+                                  np.ascontiguousarray(lb[c]), w.scale)
+
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        res = list(ex.map(one, chunks))
+    return np.concatenate([r[0] for r in res]), np.concatenate([r[1] for r in res])
 
 
 def assert_parity(out_gpu, lse_gpu, ref_out, ref_lse, what=""):
