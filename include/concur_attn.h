@@ -173,6 +173,37 @@ int concur_decode_attn_cascade(concur_attn_t* handle,
                                int32_t block_table_stride, void* cuda_stream);
 
 /*
+ * Prefill: causal attention of several new query tokens per sequence against the cache -- the
+ * step that runs once per prompt before its samples are decoded (in the paper's pipeline every
+ * task's prompt, the fixed template of App. C around the task's program, is processed once and
+ * then sampled 5 or 10 times, Sec. 3.3 / 4.1), or once per chunk of a long prompt.  The paper
+ * states no formula; per query token the definition is that of the decode step:
+ *
+ *   sequence b has q_len = q_start[b+1] - q_start[b] query tokens, rows q_start[b] .. of q, out
+ *   and lse.  They are the LAST q_len of the seq_lens[b] cached tokens (their K and V must
+ *   already be in the cache): query token i sits at position pos = seq_lens[b] - q_len + i and
+ *   attends to the cached tokens 0 .. pos of its sequence, exactly as concur_decode_attn would
+ *   for a sequence of length pos + 1.
+ *
+ *   q, out        device, bf16 [total_q][Hq][D], 16-byte aligned
+ *   lse           device, fp32 [total_q][Hq]
+ *   q_start       device, int32 [batch + 1], non-decreasing, q_start[0] = 0, q_start[batch] = total_q
+ *   other arguments as for concur_decode_attn
+ *
+ * Runs on the 5th-generation tensor cores: a unit is 16 query tokens x the query heads of one
+ * KV head (up to 128 accumulator rows in tensor memory) streaming that KV head's tiles once.
+ * Asynchronous on `cuda_stream`.  q_len > seq_lens[b] is cut to seq_lens[b] and recorded as
+ * CONCUR_FLAG_BAD_SEQ_LEN (the rows beyond are then not written).  Errors as for
+ * concur_decode_attn; total_q < 0 or a null q_start is CONCUR_ERR_INVALID_ARG.
+ */
+int concur_prefill_attn(concur_attn_t* handle,
+                        const void* q, const void* k_pages, const void* v_pages,
+                        const int32_t* block_table, const int32_t* seq_lens, const int32_t* q_start,
+                        float scale, void* out, float* lse,
+                        int32_t batch, int32_t total_q, int32_t num_pages, int32_t block_table_stride,
+                        void* cuda_stream);
+
+/*
  * The write path of the paged cache, run once per decode step before the attention call:
  * for every sequence b, the new token's rows k_new[b][g][:], v_new[b][g][:] (g = 0..Hkv-1)
  * are stored at position pos = seq_lens[b], i.e. slot pos % P of page

@@ -37,7 +37,7 @@ EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
-    "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade",
+    "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade", "concur_prefill_attn",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -75,6 +75,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_decode_attn_cascade.restype = ctypes.c_int
     lib.concur_decode_attn_cascade.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp,
                                                i32, i32, i32, i32, vp]
+    lib.concur_prefill_attn.restype = ctypes.c_int
+    lib.concur_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_kv_append.restype = ctypes.c_int
     lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
@@ -183,6 +185,17 @@ def concur_decode_attn_cascade(handle, q, k_pages, v_pages, block_table, seq_len
                                         num_pages, block_table_stride, stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_decode_attn_cascade")
+    return rc
+
+
+def concur_prefill_attn(handle, q, k_pages, v_pages, block_table, seq_lens, q_start, scale, out, lse, batch,
+                        total_q, num_pages, block_table_stride, stream=0, check=True) -> int:
+    """Causal attention of each sequence's last q_len cached tokens (device tensors)."""
+    rc = lib.concur_prefill_attn(handle, _addr(q), _addr(k_pages), _addr(v_pages), _addr(block_table),
+                                 _addr(seq_lens), _addr(q_start), ctypes.c_float(scale), _addr(out), _addr(lse),
+                                 batch, total_q, num_pages, block_table_stride, stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_prefill_attn")
     return rc
 
 

@@ -316,6 +316,32 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
     return CONCUR_OK;
 }
 
+int concur_prefill_attn(concur_attn_t* h, const void* q, const void* k_pages, const void* v_pages,
+                        const int32_t* block_table, const int32_t* seq_lens, const int32_t* q_start, float scale,
+                        void* out, float* lse, int32_t batch, int32_t total_q, int32_t num_pages,
+                        int32_t block_table_stride, void* cuda_stream) {
+    int rc = check_call(h, q, k_pages, v_pages, block_table, seq_lens, out, lse, batch, num_pages,
+                        block_table_stride, 16);
+    if (rc != CONCUR_OK || batch == 0) return rc;
+    if (total_q < 0 || !q_start || !aligned(q_start, 4)) return CONCUR_ERR_INVALID_ARG;
+    if ((int64_t)total_q * h->cfg.num_q_heads >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
+    if (total_q == 0) return CONCUR_OK;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok()) return CONCUR_ERR_CUDA;
+    DecodeParams p = {};
+    fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
+                block_table_stride);
+    p.grid_ctas = h->grid_ctas > 0 ? h->grid_ctas : h->sm_count;
+    PrefillParams f;
+    f.q_start = q_start;
+    f.total_q = total_q;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (h->ev_before && cudaEventRecord(h->ev_before, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    if (launch_prefill_tc(p, f, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    return CONCUR_OK;
+}
+
 static int ensure(Staging& s, size_t bytes) {
     if (bytes <= s.cap) return CONCUR_OK;
     if (s.ptr) cudaFree(s.ptr);

@@ -1,4 +1,6 @@
-// Prefix pass of the shared-prefix (cascade) step on the 5th-generation tensor cores.
+// Attention of many query rows against one stream of K/V tiles on the 5th-generation tensor
+// cores: the prefix pass of the shared-prefix (cascade) step and, with a causal mask, prefill.
+// The description below is written for the prefix pass; what prefill changes is listed at TCfg.
 //
 // A unit is (group, KV head): the tiles that all siblings of a group have in common.  Each
 // 64-token K/V tile is streamed from HBM once and multiplied with the query rows of all
@@ -57,8 +59,18 @@ namespace concur {
 
 namespace {
 
-constexpr int kTKStages = 5;                              // K ring: a stage is free again after Q.K^T
-constexpr int kTVStages = 6;                              // V ring: a stage is free again after P.V
+// Two uses of the same pipeline.  Prefix pass of the cascade step: a row group is a sibling (up to
+// kMaxShare = 10), every tile is whole and fully visible.  Prefill: a row group is a query token
+// (16 per unit), the tiles on the diagonal are masked causally and the last one may be ragged.
+template <bool kPrefill>
+struct TCfg {
+    static constexpr int kShare = kPrefill ? 16 : kMaxShare;          // row groups (of 8 heads) per unit
+    static constexpr int kKStages = kPrefill ? 4 : 5;                 // K ring: a stage is free again after Q.K^T
+    static constexpr int kVStages = kPrefill ? 5 : 6;                 // V ring: a stage is free again after P.V
+    static constexpr int kQRows = kShare * kGroup;                    // query rows that are really loaded
+    static constexpr int kQHalfBytes = kQRows * 128;
+    static constexpr int kQBytes = 2 * kQHalfBytes;                   // per staging buffer
+};
 constexpr int kTVLag = 2;                                 // V of tile t is requested with K of tile t + 2
 constexpr int kTMetaRing = 16;                            // tile records; readers trail the producer by < 8
 constexpr int kTProducerWarp = 8;
@@ -68,32 +80,33 @@ constexpr int kTThreads = 11 * 32;
 constexpr int kTRows = 128;                               // MMA M
 constexpr int kTHalfBytes = kTile * 128;                  // 8 KB: 64 tokens x one 64-dim half
 constexpr int kTTileBytes = 2 * kTHalfBytes;              // 16 KB: one K or V tile
-constexpr int kTQRows = kMaxShare * kGroup;               // 80 query rows that are really loaded
-constexpr int kTQHalfBytes = kTQRows * 128;               // 10 KB
-constexpr int kTQBytes = 2 * kTQHalfBytes;                // 20 KB per buffer
 // TMEM columns (512): Q as packed bf16 [0,64); S_A [64,128), S_B [128,192); P_A [192,224),
 // P_B [224,256) as packed bf16; O_A [256,384), O_B [384,512)
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemQ = 0, kTmemS = 64, kTmemP = 192, kTmemO = 256;
 
-static_assert(kTQHalfBytes % 1024 == 0, "query halves must keep the swizzle phase");
 
 struct TMeta {
-    int32_t n;            // sharing siblings (2..kMaxShare); 0 = no more work
+    int32_t n;            // live row groups (siblings / query tokens) of the segment; 0 = no more work
     int32_t idx, cnt;     // index of the tile in its segment, tiles of the segment
     int32_t qsel;         // query buffer of the segment
-    int32_t row;          // first partial row of the segment (one row per sibling)
+    int32_t row;          // prefix pass: first partial row of the segment; prefill: first query token
     int32_t g;            // KV head
     int32_t pages[4];     // physical pages of the tile (64 / P of them)
-    int32_t pad[6];
+    int32_t nvalid;       // tokens of the tile that exist and that some row may see (1..64)
+    int32_t diag;         // row group i sees columns c <= diag + i of the tile (>= 63: all of them)
+    int32_t pad[4];
 };
 static_assert(sizeof(TMeta) == 64, "one record per 64 bytes");
 
 // Shared memory, from a 1024-byte aligned base.
+template <bool kPrefill>
 struct TSmem {
+    using Cfg = TCfg<kPrefill>;
+    static constexpr int kTKStages = Cfg::kKStages, kTVStages = Cfg::kVStages;
     static constexpr int kVOff = kTKStages * kTTileBytes;
-    static constexpr int kQOff = kVOff + kTVStages * kTTileBytes;         // 2 x 20 KB staging of the queries
-    static constexpr int kXchOff = kQOff + 2 * kTQBytes;                  // [2 groups][128 rows] (m, l)
+    static constexpr int kQOff = kVOff + kTVStages * kTTileBytes;         // two staging buffers of the queries
+    static constexpr int kXchOff = kQOff + 2 * Cfg::kQBytes;              // [2 groups][128 rows] (m, l)
     static constexpr int kMetaOff = kXchOff + 2 * kTRows * 8;
     static constexpr int kBarOff = kMetaOff + kTMetaRing * (int)sizeof(TMeta);
     // full_k, empty_k per K stage; full_v, empty_v per V stage; meta_full per record; then pairs:
@@ -104,8 +117,10 @@ struct TSmem {
     static constexpr int kTotal = kAbortOff + 8;
     static constexpr int kBytes = kTotal + 1024;
 };
-static_assert(TSmem::kVOff % 1024 == 0 && TSmem::kQOff % 1024 == 0, "operand slabs must be 1024-byte aligned");
-static_assert(TSmem::kBytes <= 232448, "exceeds the 227 KB a CTA may use");
+static_assert(TSmem<false>::kQOff % 1024 == 0 && TSmem<true>::kQOff % 1024 == 0 &&
+              TCfg<false>::kQHalfBytes % 1024 == 0 && TCfg<true>::kQHalfBytes % 1024 == 0,
+              "operand slabs must be 1024-byte aligned");
+static_assert(TSmem<false>::kBytes <= 232448 && TSmem<true>::kBytes <= 232448, "exceeds the 227 KB a CTA may use");
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, int32_t c2,
                                             uint32_t bar) {
@@ -116,17 +131,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 
 }  // namespace
 
+template <bool kPrefill>
 __global__ void __launch_bounds__(kTThreads, 1)
-prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q) {
+attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q) {
+    using SM = TSmem<kPrefill>;
+    using Cfg = TCfg<kPrefill>;
+    constexpr int kTKStages = Cfg::kKStages, kTVStages = Cfg::kVStages;
+    constexpr int kTQRows = Cfg::kQRows, kTQHalfBytes = Cfg::kQHalfBytes, kTQBytes = Cfg::kQBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
-    TMeta* meta = reinterpret_cast<TMeta*>(smem + TSmem::kMetaOff);
-    float2* xch = reinterpret_cast<float2*>(smem + TSmem::kXchOff);
-    volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(smem + TSmem::kAbortOff);
-    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(smem + TSmem::kTmemPtrOff);
-    const uint32_t bar_base = smem_base + TSmem::kBarOff;
+    TMeta* meta = reinterpret_cast<TMeta*>(smem + SM::kMetaOff);
+    float2* xch = reinterpret_cast<float2*>(smem + SM::kXchOff);
+    volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(smem + SM::kAbortOff);
+    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(smem + SM::kTmemPtrOff);
+    const uint32_t bar_base = smem_base + SM::kBarOff;
     constexpr int kB0 = 2 * kTKStages + 2 * kTVStages + kTMetaRing;
     auto full_k = [&](int s) { return bar_base + 8u * s; };
     auto empty_k = [&](int s) { return bar_base + 8u * (kTKStages + s); };
@@ -150,7 +170,7 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
 
     // unused query rows must at least be defined once
     for (int i = tid; i < (2 * kTQBytes) / 16; i += kTThreads)
-        reinterpret_cast<uint4*>(smem + TSmem::kQOff)[i] = make_uint4(0, 0, 0, 0);
+        reinterpret_cast<uint4*>(smem + SM::kQOff)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int s = 0; s < kTKStages; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
         for (int s = 0; s < kTVStages; ++s) { mbar_init(full_v(s), 1); mbar_init(empty_v(s), 1); }
@@ -171,13 +191,14 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    if (warp == kTMmaWarp) tmem_alloc(smem_base + TSmem::kTmemPtrOff, kTmemCols);
+    if (warp == kTMmaWarp) tmem_alloc(smem_base + SM::kTmemPtrOff, kTmemCols);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr;
-    const int32_t W = c.chdr[kHdrTotalTiles];
-    const int32_t R = c.chdr[kHdrNumRanges];
+    // prefix pass: flat tile space and ranges of the cascade plan; prefill: W = number of units
+    const int32_t W = kPrefill ? p.hdr[kHdrTotalTiles] : c.chdr[kHdrTotalTiles];
+    const int32_t R = kPrefill ? 0 : c.chdr[kHdrNumRanges];
 
     if (warp == kTProducerWarp) {
         // =========================================================== producer warp
@@ -192,15 +213,17 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
             const int vs = u % kTVStages;
             ok = mbar_wait(empty_v(vs), ((u / kTVStages) & 1u) ^ 1u, abort_flag);
             if (!ok) return;
-            const uint32_t vdst = smem_base + TSmem::kVOff + vs * kTTileBytes;
-            mbar_arrive_expect_tx(full_v(vs), kTTileBytes);
+            const uint32_t vdst = smem_base + SM::kVOff + vs * kTTileBytes;
+            const int32_t npg = (m.nvalid + P - 1) >> p.page_shift;      // pages of the tile that are read
             if (npages == 1) {
                 // page = tile: one box {64, 64, 2} lands as [half][row][128 B], the operand layout
+                mbar_arrive_expect_tx(full_v(vs), kTTileBytes);
                 tma_load_3d(vdst, &map_v, 0, (m.pages[0] * kHkv + m.g) * P, 0, full_v(vs));
             } else {
+                mbar_arrive_expect_tx(full_v(vs), npg * 2 * page_bytes);
                 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    if (q < npages) {
+                    if (q < npg) {
                         const int32_t prow = (m.pages[q] * kHkv + m.g) * P;
                         tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(vs));
                         tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(vs));
@@ -208,90 +231,129 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
             }
             ++vt;
         };
-        int32_t r = blockIdx.x;
-        while (ok && r < R) {
-            int32_t r_next = 0;
-            if (lane == 0) r_next = atomicAdd(c.chdr + kHdrClaim, 1);
-            const int32_t x0 = range_begin(W, R, r), x1 = range_begin(W, R, r + 1);
-            int32_t x = x0;
-            while (ok && x < x1) {
-                // the prefix unit (group i, KV head g) that holds flat tile x
-                const int32_t i = find_sequence(c.ptiles_prefix, c.num_groups, x);
-                const int32_t t_i = c.ptiles_prefix[i + 1] - c.ptiles_prefix[i];
-                const int32_t base = kHkv * c.ptiles_prefix[i];
-                const int32_t g = (x - base) / t_i;
-                const int32_t unit_start = base + g * t_i;
-                const int32_t tile0 = x - unit_start;
-                const int32_t tile1 = min(x1, unit_start + t_i) - unit_start;
-                x += tile1 - tile0;
-                const int32_t b0 = c.group_start[i];
-                const int32_t n = min(c.group_start[i + 1] - b0, kMaxShare);
-                const int32_t split = r - range_of(W, R, unit_start);
-                const int32_t row = c.unit_rowbase[i * kHkv + g] + split * n;
-                const int32_t qsel = seg & 1;
-                const int32_t* table = p.block_table + (int64_t)b0 * p.bt_stride;   // the first sibling's pages
-                const int32_t page_end = tile1 << pages_per_tile_shift;
-                int32_t chunk_base = tile0 << pages_per_tile_shift;
-                int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
-                int32_t pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
-                for (int32_t t = tile0; ok && t < tile1; ++t) {
-                    const int32_t first_page = t << pages_per_tile_shift;
-                    if (first_page >= chunk_base + 32) {
-                        chunk_base += 32;
-                        pg = pg_next;
-                        pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
-                    }
-                    const int ks = it % kTKStages;
-                    int32_t my_page = __shfl_sync(0xffffffffu, pg, (first_page - chunk_base + (lane & 3)) & 31);
-                    const bool bad = (lane < npages) && (my_page < 0 || my_page >= p.num_pages);
-                    if (__any_sync(0xffffffffu, bad)) {
-                        if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagBadPage);
-                        if (my_page < 0 || my_page >= p.num_pages) my_page = 0;
-                    }
-                    const int32_t pages[4] = {__shfl_sync(0xffffffffu, my_page, 0), __shfl_sync(0xffffffffu, my_page, 1),
-                                              __shfl_sync(0xffffffffu, my_page, 2), __shfl_sync(0xffffffffu, my_page, 3)};
-                    if (lane == 0) {
-                        if (t == tile0) {
-                            // the segment's query rows: sibling j's 8 rows go to rows 8j .. 8j + 7 of both halves
-                            ok = mbar_wait(q_empty(qsel), ((seg >> 1) & 1u) ^ 1u, abort_flag);
-                            if (ok) {
-                                mbar_arrive_expect_tx(q_full(qsel), n * kGroup * kRowBytes);
-                                const uint32_t qdst = smem_base + TSmem::kQOff + qsel * kTQBytes;
-                                for (int j = 0; j < n; ++j) {
-                                    const int32_t qrow = (b0 + j) * p.hq + g * p.group;
-                                    tma_load_3d(qdst + j * 1024, &map_q, 0, qrow, 0, q_full(qsel));
-                                    tma_load_3d(qdst + kTQHalfBytes + j * 1024, &map_q, 0, qrow, 1, q_full(qsel));
-                                }
-                            }
-                        }
-                        if (ok) ok = mbar_wait(empty_k(ks), ((it / kTKStages) & 1u) ^ 1u, abort_flag);
-                        if (ok) {
-                            TMeta& m = meta[it % kTMetaRing];
-                            m.n = n; m.idx = t - tile0; m.cnt = tile1 - tile0; m.qsel = qsel; m.row = row; m.g = g;
-                            m.pages[0] = pages[0]; m.pages[1] = pages[1]; m.pages[2] = pages[2]; m.pages[3] = pages[3];
-                            mbar_arrive(meta_full(it % kTMetaRing));
-                            const uint32_t kdst = smem_base + ks * kTTileBytes;
-                            mbar_arrive_expect_tx(full_k(ks), kTTileBytes);
-                            if (npages == 1) {
-                                tma_load_3d(kdst, &map_k, 0, (pages[0] * kHkv + g) * P, 0, full_k(ks));
-                            } else {
-                                #pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    if (q < npages) {
-                                        const int32_t prow = (pages[q] * kHkv + g) * P;
-                                        tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
-                                        tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
-                                    }
-                            }
-                            if (it >= (uint32_t)kTVLag) issue_v(it - kTVLag);
-                        }
-                    }
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (ok) ++it;
+        // One segment: tiles [tile0, tile1) of KV head g through the table row `table`, for `n` row
+        // groups whose query rows are (qbase + j) * Hq + g * G.  pos0 / pos_last: positions of the
+        // first and last row group (prefill; the prefix pass sees every token of its tiles).
+        auto stream_segment = [&](const int32_t* table, int32_t g, int32_t tile0, int32_t tile1, int32_t n,
+                                  int32_t row, int32_t qbase, int32_t pos0, int32_t pos_last) {
+            const int32_t qsel = seg & 1;
+            const int32_t tok_end = min(tile1 * kTile, pos_last + 1);
+            const int32_t page_end = (tok_end + P - 1) >> p.page_shift;
+            int32_t chunk_base = tile0 << pages_per_tile_shift;
+            int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
+            int32_t pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
+            for (int32_t t = tile0; ok && t < tile1; ++t) {
+                const int32_t first_page = t << pages_per_tile_shift;
+                if (first_page >= chunk_base + 32) {
+                    chunk_base += 32;
+                    pg = pg_next;
+                    pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                 }
-                ++seg;
+                const int32_t nvalid = min(kTile, tok_end - t * kTile);
+                const int32_t npg = (nvalid + P - 1) >> p.page_shift;          // pages of the tile that are read
+                const int ks = it % kTKStages;
+                int32_t my_page = __shfl_sync(0xffffffffu, pg, (first_page - chunk_base + (lane & 3)) & 31);
+                const bool bad = (lane < npg) && (my_page < 0 || my_page >= p.num_pages);
+                if (__any_sync(0xffffffffu, bad)) {
+                    if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagBadPage);
+                    if (my_page < 0 || my_page >= p.num_pages) my_page = 0;
+                }
+                const int32_t pages[4] = {__shfl_sync(0xffffffffu, my_page, 0), __shfl_sync(0xffffffffu, my_page, 1),
+                                          __shfl_sync(0xffffffffu, my_page, 2), __shfl_sync(0xffffffffu, my_page, 3)};
+                if (lane == 0) {
+                    if (t == tile0) {
+                        // the segment's query rows: row group j's 8 rows go to rows 8j .. 8j + 7 of both halves
+                        ok = mbar_wait(q_empty(qsel), ((seg >> 1) & 1u) ^ 1u, abort_flag);
+                        if (ok) {
+                            mbar_arrive_expect_tx(q_full(qsel), n * kGroup * kRowBytes);
+                            const uint32_t qdst = smem_base + SM::kQOff + qsel * kTQBytes;
+                            for (int j = 0; j < n; ++j) {
+                                const int32_t qrow = (qbase + j) * p.hq + g * p.group;
+                                tma_load_3d(qdst + j * 1024, &map_q, 0, qrow, 0, q_full(qsel));
+                                tma_load_3d(qdst + kTQHalfBytes + j * 1024, &map_q, 0, qrow, 1, q_full(qsel));
+                            }
+                        }
+                    }
+                    if (ok) ok = mbar_wait(empty_k(ks), ((it / kTKStages) & 1u) ^ 1u, abort_flag);
+                    if (ok) {
+                        TMeta& m = meta[it % kTMetaRing];
+                        m.n = n; m.idx = t - tile0; m.cnt = tile1 - tile0; m.qsel = qsel; m.row = row; m.g = g;
+                        m.pages[0] = pages[0]; m.pages[1] = pages[1]; m.pages[2] = pages[2]; m.pages[3] = pages[3];
+                        m.nvalid = nvalid;
+                        m.diag = kPrefill ? min(pos0 - t * kTile, 1 << 20) : (1 << 20);
+                        mbar_arrive(meta_full(it % kTMetaRing));
+                        const uint32_t kdst = smem_base + ks * kTTileBytes;
+                        if (npages == 1) {
+                            mbar_arrive_expect_tx(full_k(ks), kTTileBytes);
+                            tma_load_3d(kdst, &map_k, 0, (pages[0] * kHkv + g) * P, 0, full_k(ks));
+                        } else {
+                            mbar_arrive_expect_tx(full_k(ks), npg * 2 * page_bytes);
+                            #pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                if (q < npg) {
+                                    const int32_t prow = (pages[q] * kHkv + g) * P;
+                                    tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
+                                    tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
+                                }
+                        }
+                        if (it >= (uint32_t)kTVLag) issue_v(it - kTVLag);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (ok) ++it;
             }
-            r = __shfl_sync(0xffffffffu, r_next, 0);
+            ++seg;
+        };
+        int32_t r = blockIdx.x;
+        if constexpr (!kPrefill) {
+            while (ok && r < R) {
+                int32_t r_next = 0;
+                if (lane == 0) r_next = atomicAdd(c.chdr + kHdrClaim, 1);
+                const int32_t x0 = range_begin(W, R, r), x1 = range_begin(W, R, r + 1);
+                int32_t x = x0;
+                while (ok && x < x1) {
+                    // the prefix unit (group i, KV head g) that holds flat tile x
+                    const int32_t i = find_sequence(c.ptiles_prefix, c.num_groups, x);
+                    const int32_t t_i = c.ptiles_prefix[i + 1] - c.ptiles_prefix[i];
+                    const int32_t base = kHkv * c.ptiles_prefix[i];
+                    const int32_t g = (x - base) / t_i;
+                    const int32_t unit_start = base + g * t_i;
+                    const int32_t tile0 = x - unit_start;
+                    const int32_t tile1 = min(x1, unit_start + t_i) - unit_start;
+                    x += tile1 - tile0;
+                    const int32_t b0 = c.group_start[i];
+                    const int32_t n = min(c.group_start[i + 1] - b0, kMaxShare);
+                    const int32_t split = r - range_of(W, R, unit_start);
+                    const int32_t row = c.unit_rowbase[i * kHkv + g] + split * n;
+                    // shared tiles are whole; they are read through the first sibling's table row
+                    stream_segment(p.block_table + (int64_t)b0 * p.bt_stride, g, tile0, tile1, n, row, b0,
+                                   1 << 28, tile1 * kTile - 1);
+                }
+                r = __shfl_sync(0xffffffffu, r_next, 0);
+            }
+        } else {
+            // prefill: unit r = (sequence b, block of 16 query tokens, KV head g); the blocks of a
+            // sequence are taken last first (they have the most tiles); a unit is never split
+            const int64_t max_len = (int64_t)p.bt_stride * P;
+            while (ok && r < W) {
+                int32_t r_next = 0;
+                if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
+                const int32_t b = find_sequence(p.tiles_prefix, p.batch, r);
+                const int32_t local = r - kHkv * p.tiles_prefix[b];
+                const int32_t nqb = p.tiles_prefix[b + 1] - p.tiles_prefix[b];
+                const int32_t qb = nqb - 1 - local / kHkv, g = local % kHkv;
+                int64_t len = p.seq_lens[b];
+                len = len < 0 ? 0 : (len > max_len ? max_len : len);
+                int32_t q_len = f.q_start[b + 1] - f.q_start[b];
+                if (q_len > (int32_t)len) q_len = (int32_t)len;                 // flagged by the plan
+                const int32_t tok0 = qb * Cfg::kShare;
+                const int32_t n = min(Cfg::kShare, q_len - tok0);
+                const int32_t pos0 = (int32_t)len - q_len + tok0;
+                const int32_t pos_last = pos0 + n - 1;
+                stream_segment(p.block_table + (int64_t)b * p.bt_stride, g, 0, pos_last / kTile + 1, n,
+                               f.q_start[b] + tok0, f.q_start[b] + tok0, pos0, pos_last);
+                r = __shfl_sync(0xffffffffu, r_next, 0);
+            }
         }
         if (lane == 0) {
             while (ok && vt < it) issue_v(vt);                 // the last tiles' V
@@ -356,32 +418,49 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
         }
         __syncwarp();
     } else if (warp == kTPvWarp) {
-        // =========================================================== P.V warp (one thread issues)
-        if (lane == 0) {
+        // =========================================================== P.V warp (one lane issues)
+        {
             constexpr uint32_t idesc_pv = umma_idesc_bf16(kTRows, kD, false, true);
             bool ok = true;
             int site = 0;
             for (uint32_t u = 0; ok; ++u) {
                 const int g = u & 1u;
                 if (!mbar_wait(meta_full(u % kTMetaRing), (u / kTMetaRing) & 1u, abort_flag)) { ok = false; site = 46; break; }
-                const TMeta mt = meta[u % kTMetaRing];
-                if (mt.n == 0) break;
+                const TMeta* mt = &meta[u % kTMetaRing];
+                const int32_t idx = mt->idx, nvalid = mt->nvalid;
+                if (mt->n == 0) break;
                 const int vs = u % kTVStages;
                 if (!mbar_wait(p_full(g), (u >> 1) & 1u, abort_flag)) { ok = false; site = 35; break; }
                 if (!mbar_wait(full_v(vs), (u / kTVStages) & 1u, abort_flag)) { ok = false; site = 36; break; }
-                tc_fence_after_sync();
-                const uint32_t v_addr = smem_base + TSmem::kVOff + vs * kTTileBytes;
-                #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t b = umma_smem_desc(v_addr + kk * 2048, kTHalfBytes, 1024);
-                    // a group's first tile of a segment overwrites its accumulator
-                    umma_ts(tmem_base + kTmemO + g * kD, tmem_base + kTmemP + g * 32 + kk * 8, b, idesc_pv,
-                            (mt.idx < 2 && kk == 0) ? 0u : 1u);
+                const uint32_t v_addr = smem_base + SM::kVOff + vs * kTTileBytes;
+                if (nvalid < kTile) {
+                    // rows past the last token may hold anything (NaN included, or another tile's data
+                    // where no page was read) and a zero probability does not silence them inside an
+                    // MMA: clear them in both halves first
+                    for (int i = lane; i < (kTile - nvalid) * 16; i += 32) {
+                        const int rowi = nvalid + (i >> 4), c16 = i & 15;
+                        const uint32_t addr = v_addr + (uint32_t)(c16 >> 3) * kTHalfBytes + (uint32_t)rowi * 128u +
+                                              (uint32_t)((c16 & 7) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
                 }
-                umma_commit(empty_v(vs));               // that V stage may be overwritten
-                umma_commit(pv_done(g));
+                tc_fence_after_sync();
+                if (lane == 0) {
+                    #pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint64_t b = umma_smem_desc(v_addr + kk * 2048, kTHalfBytes, 1024);
+                        // a group's first tile of a segment overwrites its accumulator
+                        umma_ts(tmem_base + kTmemO + g * kD, tmem_base + kTmemP + g * 32 + kk * 8, b, idesc_pv,
+                                (idx < 2 && kk == 0) ? 0u : 1u);
+                    }
+                    umma_commit(empty_v(vs));               // that V stage may be overwritten
+                    umma_commit(pv_done(g));
+                }
+                __syncwarp();
             }
-            if (!ok) wait_failed(p, abort_flag, site);
+            if (!ok && lane == 0) wait_failed(p, abort_flag, site);
         }
         __syncwarp();
     } else {
@@ -417,7 +496,7 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                     if (!mbar_wait(qt_free, (qsegs - 1) & 1u, abort_flag)) { ok = false; site = 45; break; }
                     tc_fence_after_sync();
                 }
-                const uint8_t* qsrc = smem + TSmem::kQOff + mt.qsel * kTQBytes + row * 128;
+                const uint8_t* qsrc = smem + SM::kQOff + mt.qsel * kTQBytes + row * 128;
                 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint32_t qw[32];
@@ -449,9 +528,23 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                     tmem_wait_ld();
                     tc_fence_before_sync();
                     mbar_arrive(s_free(g));
+                    float scl = sc;                              // what the values in raw[] still have to be multiplied by
+                    bool neg = sc_neg;
+                    if (kPrefill && mt.diag + j < kTile - 1) {
+                        // causal diagonal (or ragged last tile): this row sees columns 0 .. diag + j only.
+                        // Scale first, then replace what is hidden by -inf with a select: hidden K rows
+                        // may hold anything.
+                        const int limit = mt.diag + j;
+                        #pragma unroll
+                        for (int e = 0; e < 64; ++e) {
+                            const float v = __uint_as_float(raw[e >> 5][e & 31]) * sc;
+                            raw[e >> 5][e & 31] = __float_as_uint(e <= limit ? v : -INFINITY);
+                        }
+                        scl = 1.f; neg = false;
+                    }
                     // extreme raw score of the tile (two chains); the scale may be negative
                     float e0 = __uint_as_float(raw[0][0]), e1 = __uint_as_float(raw[1][0]);
-                    if (!sc_neg) {
+                    if (!neg) {
                         #pragma unroll
                         for (int e = 1; e < 31; e += 2) {
                             asm("max.f32 %0, %0, %1, %2;" : "+f"(e0) : "f"(__uint_as_float(raw[0][e])), "f"(__uint_as_float(raw[0][e + 1])));
@@ -468,17 +561,17 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                         asm("min.f32 %0, %0, %1, %2;" : "+f"(e0) : "f"(__uint_as_float(raw[0][31])), "f"(__uint_as_float(raw[1][31])));
                         e0 = fminf(e0, e1);
                     }
-                    const float mx = e0 * sc;
+                    const float mx = e0 * scl;
                     need = !first && (mx > m_ref + kSlack);
                     m_use = (first || need) ? mx : m_ref;
                     if (need) alpha = fast_exp2(m_ref - mx);
-                    const float neg_m = -m_use;
+                    const float neg_m = (m_use == -INFINITY) ? 0.f : -m_use;   // a row that sees nothing yet: P = 0
                     float sum1 = 0.f;
                     #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const int t0 = 2 * e;
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(raw[t0 >> 5][t0 & 31]), sc, neg_m));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(raw[(t0 + 1) >> 5][(t0 + 1) & 31]), sc, neg_m));
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(raw[t0 >> 5][t0 & 31]), scl, neg_m));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(raw[(t0 + 1) >> 5][(t0 + 1) & 31]), scl, neg_m));
                         sum += p0; sum1 += p1;
                         pk[e] = pack_bf16(p0, p1);
                     }
@@ -529,22 +622,42 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                 if (!mbar_wait(xch_a, segs & 1u, abort_flag)) { ok = false; site = 41; break; }
                 if (warp_live) {
                     const float2 other = xch[(g ^ 1) * kTRows + row];
-                    const bool had2 = other.y > 0.f;
+                    // Whether the other group took a tile of this segment is the same for every row
+                    // (the TMEM loads below are warp-wide instructions and may depend on nothing
+                    // else); whether a particular row of it saw any token is not, and is a select.
+                    const bool had_other = !mine || mt.cnt >= 2;
+                    const bool had2 = had_other && other.y > 0.f;
                     const float m1 = had ? m_ref : -INFINITY, l1 = had ? l : 0.f;
                     const float M = fmaxf(m1, other.x);
                     const float w1 = had ? fast_exp2(m1 - M) : 0.f, w2 = had2 ? fast_exp2(other.x - M) : 0.f;
                     const float L = l1 * w1 + other.y * w2;
                     const float inv = 1.f / L;
                     const float f1 = w1 * inv, f2 = w2 * inv;
-                    const bool live = j < mt.n;
+                    // prefix pass: a normalised fp32 partial per sibling; prefill: the final rows of out / lse
+                    const bool live = j < mt.n && (!kPrefill || head < p.group);
                     float* dst = c.pre_o + ((int64_t)(mt.row + j) * kGroup + head) * kD + g * 64;
+                    const int64_t out_row = (int64_t)(mt.row + j) * p.hq + mt.g * p.group + head;
                     #pragma unroll
                     for (int cblk = 0; cblk < 2; ++cblk) {
                         uint32_t oa[32], ob[32];
                         if (had) tmem_ld32(o_mine + g * 64 + cblk * 32, oa);
-                        if (had2) tmem_ld32(o_other + g * 64 + cblk * 32, ob);
+                        if (had_other) tmem_ld32(o_other + g * 64 + cblk * 32, ob);
                         tmem_wait_ld();
-                        if (live) {
+                        if (kPrefill && live) {
+                            uint4* od = reinterpret_cast<uint4*>(p.out + out_row * kD + g * 64 + cblk * 32);
+                            #pragma unroll
+                            for (int e = 0; e < 32; e += 8) {
+                                float v[8];
+                                #pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    const float a = had ? __uint_as_float(oa[e + q]) * f1 : 0.f;
+                                    v[q] = had2 ? fmaf(__uint_as_float(ob[e + q]), f2, a) : a;
+                                }
+                                od[e >> 3] = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
+                                                        pack_bf16(v[6], v[7]));
+                            }
+                        }
+                        if (!kPrefill && live) {
                             #pragma unroll
                             for (int e = 0; e < 32; e += 4) {
                                 float4 v;
@@ -558,7 +671,10 @@ prefix_tc_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUtens
                             }
                         }
                     }
-                    if (live && g == 0) c.pre_lse[(int64_t)(mt.row + j) * kGroup + head] = M + log2f(L);
+                    if (live && g == 0) {
+                        if (kPrefill) p.lse[out_row] = (M + log2f(L)) * 0.6931471805599453f;
+                        else c.pre_lse[(int64_t)(mt.row + j) * kGroup + head] = M + log2f(L);
+                    }
                 }
                 // nobody's next P.V may overwrite an accumulator the other group is still reading
                 tc_fence_before_sync();
@@ -615,21 +731,91 @@ bool make_half_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
-
-cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
+template <bool kPrefill>
+cudaError_t launch_attn_tc(const DecodeParams& p, const CascadeParams& c, const PrefillParams& f, uint64_t q_rows,
+                           int grid, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
     const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
     // a 64-token page is a whole tile: both halves come with one copy ([half][row][128 B])
     const uint32_t halves = p.page_size == kTile ? 2 : 1;
     if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.page_size, halves) ||
         !make_half_row_map(&mv, p.v_pages, pool_rows, p.page_size, halves) ||
-        !make_half_row_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup))
+        !make_half_row_map(&mq, p.q, q_rows, kGroup))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TSmem::kBytes);
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<kPrefill>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TSmem<kPrefill>::kBytes);
     if (e != cudaSuccess) return e;
-    prefix_tc_kernel<<<c.grid_ctas, kTThreads, TSmem::kBytes, stream>>>(p, c, mk, mv, mq);
+    attn_tc_kernel<kPrefill><<<grid, kTThreads, TSmem<kPrefill>::kBytes, stream>>>(p, c, f, mk, mv, mq);
     return cudaGetLastError();
+}
+
+constexpr int kPrefillPlanThreads = 1024;
+
+}  // namespace
+
+cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
+    return launch_attn_tc<false>(p, c, PrefillParams{}, (uint64_t)p.batch * p.hq, c.grid_ctas, stream);
+}
+
+// ---- prefill plan: blocks of 16 query tokens per sequence and their prefix sums; one unit per
+//      (sequence, block, KV head)
+__global__ void __launch_bounds__(kPrefillPlanThreads) plan_prefill_kernel(DecodeParams p, PrefillParams f) {
+    __shared__ int32_t warp_sums[kPrefillPlanThreads / 32];
+    __shared__ int32_t carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) { carry_s = 0; p.tiles_prefix[0] = 0; }
+    __syncthreads();
+    const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
+    uint32_t flags = 0;
+    for (int base = 0; base < p.batch; base += kPrefillPlanThreads) {
+        const int b = base + tid;
+        int32_t blocks = 0;
+        if (b < p.batch) {
+            int64_t len = p.seq_lens[b];
+            if (len < 0) { len = 0; flags |= kFlagBadLen; }
+            if (len > max_len) { len = max_len; flags |= kFlagBadLen; }
+            int64_t q_len = (int64_t)f.q_start[b + 1] - f.q_start[b];
+            if (q_len < 0) { q_len = 0; flags |= kFlagBadLen; }
+            if (q_len > len) { q_len = len; flags |= kFlagBadLen; }      // more query tokens than cached tokens
+            blocks = (int32_t)((q_len + TCfg<true>::kShare - 1) / TCfg<true>::kShare);
+        }
+        int32_t v = blocks;
+        #pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t n = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += n;
+        }
+        if (lane == 31) warp_sums[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t w = warp_sums[lane];
+            #pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t n = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += n;
+            }
+            warp_sums[lane] = w;
+        }
+        __syncthreads();
+        const int32_t incl = v + (warp ? warp_sums[warp - 1] : 0) + carry_s;
+        if (b < p.batch) p.tiles_prefix[b + 1] = incl;
+        __syncthreads();
+        if (tid == kPrefillPlanThreads - 1) carry_s = incl;
+        __syncthreads();
+    }
+    if (flags) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), flags);
+    if (tid == 0) {
+        p.hdr[kHdrTotalTiles] = kHkv * carry_s;          // units
+        p.hdr[kHdrNumRanges] = kHkv * carry_s;
+        p.hdr[kHdrClaim] = p.grid_ctas;
+    }
+}
+
+cudaError_t launch_prefill_tc(const DecodeParams& p, const PrefillParams& f, cudaStream_t stream) {
+    plan_prefill_kernel<<<1, kPrefillPlanThreads, 0, stream>>>(p, f);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_attn_tc<true>(p, CascadeParams{}, f, (uint64_t)f.total_q * p.hq, p.grid_ctas, stream);
 }
 
 }  // namespace concur

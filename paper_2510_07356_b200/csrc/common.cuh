@@ -85,6 +85,12 @@ struct CascadeParams {
     float* pre_lse;               // [max_rows][kGroup]     their base-2 log-sum-exp
 };
 
+// Prefill (several query tokens per sequence, causal).  Device pointer.
+struct PrefillParams {
+    const int32_t* q_start;       // [batch + 1] first query token of each sequence in q / out; last entry = total_q
+    int32_t total_q;
+};
+
 // First flat tile of range r when [0, W) is cut into R ranges of equal size.
 __device__ __forceinline__ int32_t range_begin(int32_t W, int32_t R, int32_t r) {
     return (int32_t)(((int64_t)W * r) / R);
@@ -157,6 +163,7 @@ cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_plan_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
+cudaError_t launch_prefill_tc(const DecodeParams& p, const PrefillParams& f, cudaStream_t stream);
 cudaError_t launch_combine_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 int partial_scalar_ctas_per_sm();
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,

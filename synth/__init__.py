@@ -359,3 +359,64 @@ def cascade_prefix_bytes(cw: CascadeWorkload) -> int:
         if n >= 2:
             total += (int(pre) // 64) * 64 * per_token + n * s.num_q_heads * s.head_dim * 2
     return total
+
+
+@dataclass
+class PrefillWorkload:
+    """A paged cache plus, per sequence, the query rows of its last `q_lens[b]` cached tokens."""
+    w: Workload                    # w.q is [total_q][Hq][D] here
+    q_start: torch.Tensor          # [B + 1] int32
+    q_start_host: np.ndarray = field(default=None)
+
+    @property
+    def total_q(self) -> int:
+        return int(self.q_start_host[-1])
+
+    def flops(self) -> int:
+        """Multiply-adds x 2 of the causal products: every query row against the tokens it sees,
+        for Q.K^T and for P.V."""
+        s = self.w.spec
+        total = 0
+        for b in range(s.batch):
+            n, ql = int(self.w.lens_host[b]), int(self.q_start_host[b + 1] - self.q_start_host[b])
+            seen = ql * (n - ql) + ql * (ql + 1) // 2       # tokens visible to the ql query tokens together
+            total += seen * s.num_q_heads * s.head_dim * 2 * 2
+        return total
+
+
+def make_prefill_workload(name, lens, q_lens, page_size, seed, device="cpu", num_q_heads=NUM_Q_HEADS,
+                          q_std=1.0) -> PrefillWorkload:
+    """Sequences of `lens` cached tokens whose last `q_lens` tokens are the query tokens
+    (q_lens[b] <= lens[b]; q_lens == lens is the prefill of a whole prompt, smaller values a
+    chunk of it).  Pools, tables and poisoning as in make_workload; q ~ N(0, q_std^2)."""
+    spec = tiny_spec(name, [int(x) for x in lens], page_size, seed, num_q_heads=num_q_heads, q_std=q_std)
+    w = make_workload(spec, device)
+    qs = np.zeros(len(lens) + 1, dtype=np.int32)
+    qs[1:] = np.cumsum(np.asarray(q_lens, dtype=np.int64))
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed * 1000 + 9)
+    w.q = _normal_bf16((max(int(qs[-1]), 1), num_q_heads, spec.head_dim), q_std, g, dev)[:int(qs[-1])]
+    return PrefillWorkload(w=w, q_start=torch.from_numpy(qs).to(dev), q_start_host=qs)
+
+
+def prefill_as_decode(pw: PrefillWorkload, tokens) -> Workload:
+    """Host-side restatement of some query tokens of a prefill workload as a decode batch: query
+    token t of sequence b becomes a 'sequence' with b's block-table row and length position + 1.
+    (Index bookkeeping only: what is computed per row is then the plain decode definition.)"""
+    w = pw.w
+    tokens = [int(t) for t in tokens]
+    rows, lens = [], []
+    for t in tokens:
+        b = int(np.searchsorted(pw.q_start_host, t, side="right") - 1)
+        ql = int(pw.q_start_host[b + 1] - pw.q_start_host[b])
+        pos = int(w.lens_host[b]) - ql + (t - int(pw.q_start_host[b]))
+        rows.append(w.table_host[b]); lens.append(pos + 1)
+    lens = np.asarray(lens, dtype=np.int32)
+    table = np.stack(rows).astype(np.int32) if rows else np.zeros((0, w.table_host.shape[1]), np.int32)
+    spec = Spec(w.spec.name + "_as_decode", len(lens), w.spec.page_size, ("list", [int(x) for x in lens]),
+                seed=w.spec.seed, num_q_heads=w.spec.num_q_heads)
+    idx = torch.as_tensor(tokens, dtype=torch.long)
+    return Workload(spec=spec, q=w.q.cpu()[idx], k_pages=w.k_pages.cpu(), v_pages=w.v_pages.cpu(),
+                    block_table=torch.from_numpy(table), seq_lens=torch.from_numpy(lens), scale=w.scale,
+                    lens_host=lens, table_host=table)
