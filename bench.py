@@ -5,7 +5,8 @@ C ABI on seeded synthetic long-trace workloads.
 
 NAME is one of synth.SPECS (plain decode step; the default is the 64 x 16,384 configuration) or of
 synth.CASCADE_SPECS (shared-prefix step: `value` counts the shared pages once, `logical_gbs` as if
-every sequence had read its whole context, `roofline` is the prefix-pass kernel).
+every sequence had read its whole context, `roofline` is the prefix-pass kernel) or of
+synth.PREFILL_SPECS (causal prefill: `value` is useful TFLOP/s against the measured bf16 tensor peak).
 
 One JSON line on stdout (rank 0).  `value` is the algorithmic bytes of the step (K and V of
 every cached token, q/out/lse, used table entries) divided by the device time of the whole
@@ -374,6 +375,106 @@ def run_cascade(args):
         dist.destroy_process_group()
 
 
+def measured_tensor_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def run_prefill(args):
+    """Causal prefill attention on a named prefill workload (1 GPU or replicas): useful TFLOP/s."""
+    import torch
+    import torch.distributed as dist
+    import synth
+    import paper_2510_07356_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    pw = synth.make_named_prefill(args.workload, dev)
+    w, spec = pw.w, pw.w.spec
+    attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
+    tq = pw.total_q
+    out = torch.empty((tq, spec.num_q_heads, spec.head_dim), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((tq, spec.num_q_heads), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        P.concur_prefill_attn(attn.handle, w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, pw.q_start,
+                              w.scale, out, lse, spec.batch, tq, w.num_pages, w.block_table.shape[1],
+                              stream.cuda_stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    K = args.steps
+    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)     # the caches fit in L2
+    for _ in range(max(3, args.warmup)):
+        flush_buf.zero_()
+        step()
+    barrier()
+    assert attn.status() == 0, "device-side flags set during warm-up"
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+    barrier()
+    t_mark0 = time.time()
+    for i in range(K):
+        flush_buf.zero_()
+        ev[i][0].record(stream)
+        step()
+        ev[i][1].record(stream)
+    barrier()
+    t_mark1 = time.time()
+    clocks = sampler.stop(t_mark0, t_mark1) if rank == 0 else None
+    step_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
+    ms_per_step = over_ranks([sum(step_ms) / K], "max", dev)[0]
+    flops = pw.flops()
+    job_flops, job_q = over_ranks([flops, tq], "sum", dev)
+    flags = attn.status()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_tensor_peak()
+    value = job_flops / (ms_per_step * 1e-3) / 1e12
+    line = {
+        "metric": "prefill_attention_useful_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "prompts": spec.batch, "query_tokens": tq, "kv_tokens": w.kv_tokens,
+                   "page_size": spec.page_size, "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128,
+                   "causal_flops": flops, "l2": "flushed between steps", "entry": "concur_prefill_attn",
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+        "query_tokens_per_s": job_q / (ms_per_step * 1e-3),
+        "roofline": {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s",
+                     "frac": value / world / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "kernel": "plan + attn_tc_kernel<prefill>", "ms": ms_per_step, "ms_min": min(step_ms)},
+        "e2e": None, "gpu_launches": 2 * K, "clocks": clocks, "device_flags": flags,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -381,6 +482,9 @@ def main():
         return
     if args.workload.startswith("casc"):
         run_cascade(args)
+        return
+    if args.workload.startswith("prefill"):
+        run_prefill(args)
         return
 
     import torch

@@ -420,3 +420,19 @@ def prefill_as_decode(pw: PrefillWorkload, tokens) -> Workload:
     return Workload(spec=spec, q=w.q.cpu()[idx], k_pages=w.k_pages.cpu(), v_pages=w.v_pages.cpu(),
                     block_table=torch.from_numpy(table), seq_lens=torch.from_numpy(lens), scale=w.scale,
                     lens_host=lens, table_host=table)
+
+
+# Prefill workloads: (prompts, prompt tokens, query tokens per prompt, page size, seed).  The first is
+# shaped like the paper's prompts (one fixed template around a task's program, one or two thousand
+# tokens, prefilled whole); the others are longer prompts and a chunk at the end of a long context.
+PREFILL_SPECS = {
+    "prefill_16x2048_p64": (16, 2048, 2048, 64, 73581),
+    "prefill_4x8192_p64": (4, 8192, 8192, 64, 73582),
+    "prefill_2x32768_p64": (2, 32768, 32768, 64, 73583),
+    "prefill_chunk_8x2048_of_16384_p64": (8, 16384, 2048, 64, 73584),
+}
+
+
+def make_named_prefill(name: str, device="cpu") -> PrefillWorkload:
+    prompts, n, ql, page_size, seed = PREFILL_SPECS[name]
+    return make_prefill_workload(name, [n] * prompts, [ql] * prompts, page_size, seed, device)
