@@ -435,6 +435,9 @@ def run_prefill(args):
         sampler.start()
         time.sleep(0.2)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+    for row in ev:                       # materialise the cudaEvent_t handles outside the timed region
+        for e in row:
+            e.record(stream)
     barrier()
     t_mark0 = time.time()
     for i in range(K):
