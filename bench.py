@@ -478,6 +478,97 @@ def run_prefill(args):
         dist.destroy_process_group()
 
 
+def run_curate(args):
+    """The curation arithmetic on the synthesis-run-shaped record table (rank 0 only; the job is
+    tiny and does not shard)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    import torch
+    import paper_2510_07356_b200 as P
+    from synth import records as R
+    B = P.binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    rec = R.make_records()
+    N, M = rec.correct.shape
+    host = [rec.correct, rec.t_torch, rec.t_kernel, rec.length, rec.sample_key, rec.task_key]
+    pinned = [torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in host]
+    ins = [t.to(dev) for t in pinned]
+    outs = [torch.empty((N, M), device=dev), torch.empty((N,), dtype=torch.int32, device=dev),
+            torch.empty((N, M), dtype=torch.uint8, device=dev), torch.empty((4, N), dtype=torch.int32, device=dev),
+            torch.empty((4, N), dtype=torch.uint8, device=dev), torch.empty((N,), dtype=torch.uint8, device=dev),
+            torch.empty((B.CONCUR_CURATE_NUM_STATS,), dtype=torch.float64, device=dev)]
+    prm = B.concur_curate_params_t(N, M, 5.0, 1.0, 4892, 4000, 8500, 0)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        B.concur_curate(prm, *ins, *outs, stream.cuda_stream)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize(dev)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = "0"
+    sampler = ClockSampler(gpu_id)
+    sampler.start(); time.sleep(0.2)
+    K = args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream); e1.record(stream); torch.cuda.synchronize(dev)
+    t0m = time.time()
+    e0.record(stream)
+    for _ in range(K):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / K
+    # end to end: records from pinned host memory, the statistics and the rule (a) picks read back
+    stats_h = torch.empty(B.CONCUR_CURATE_NUM_STATS, dtype=torch.float64).pin_memory()
+    rule_a_h = torch.empty(N, dtype=torch.int32).pin_memory()
+    e0.record(stream)
+    for _ in range(K):
+        for d, h in zip(ins, pinned):
+            d.copy_(h, non_blocking=True)
+        step()
+        stats_h.copy_(outs[6], non_blocking=True); rule_a_h.copy_(outs[1], non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    e2e_ms = e0.elapsed_time(e1) / K
+    clocks = sampler.stop(t0m, time.time())
+    # CPU baseline: the oracle, as it stands, on the whole table
+    from oracle import curation as C
+    t0 = time.perf_counter()
+    sp = C.speedup(rec.correct, rec.t_torch, rec.t_kernel)
+    C.rule_a(rec.correct, sp, rec.length); C.rule_b(sp); C.difficulty(rec.length); C.pearson(rec.length, sp, rec.correct)
+    C.select_random(rec.correct, rec.sample_key, rec.task_key, 4892); C.select_max_length(rec.correct, rec.length, 4892)
+    C.select_min_length(rec.correct, rec.length, 4892); C.select_speedup(rec.correct, sp, 4892)
+    cpu_s = time.perf_counter() - t0
+    records = N * M
+    # the counting rank dominates: 4 selections x N^2 (key, index) comparisons of about 4 lane
+    # operations each, against 148 SMs x 128 lanes at the sampled SM clock
+    comparisons = 4.0 * N * N
+    mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    alu_peak = 148 * 128 * mhz * 1e6 / 4.0
+    line = {"metric": "curation_records_per_s", "value": records / (ms * 1e-3), "unit": "records/s", "n_gpus": 1,
+            "steps": K, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "replicas only", "vs_baseline": None, "dtype": "f32/f64/int32", "data": "synthetic",
+            "config": {"workload": "curate_18162x5", "tasks": N, "generations": M, "top_k": 4892},
+            "roofline": {"bound": "alu", "achieved": comparisons / (ms * 1e-3), "peak": alu_peak,
+                         "unit": "rank comparisons/s", "frac": comparisons / (ms * 1e-3) / alu_peak, "traffic": None,
+                         "kernel": "curate_rank_kernel (whole call timed; it is > 90 % of it)"},
+            "e2e": {"value": records / (e2e_ms * 1e-3), "unit": "records/s", "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in pinned)),
+                    "d2h_bytes_per_step": int(stats_h.numel() * 8 + rule_a_h.numel() * 4), "entry": "concur_curate"},
+            "cpu_baseline": {"value": records / cpu_s, "unit": "records/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the whole table once, {cpu_s:.1f} s"},
+            "gpu_launches": 3 * K, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -488,6 +579,9 @@ def main():
         return
     if args.workload.startswith("prefill"):
         run_prefill(args)
+        return
+    if args.workload.startswith("curate"):
+        run_curate(args)
         return
 
     import torch

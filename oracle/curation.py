@@ -22,7 +22,8 @@ Readings where the text is silent: ties in "shortest" / "longest" / "highest" go
 generation index; rule (a) needs the shortest generation to be correct (an incorrect one has
 speedup 0 and nothing to add to a dataset) and "highest" means >= every other generation's
 speedup; tasks that tie in a ranking go by lower task index; the random selection draws no
-numbers itself -- it ranks by keys that the caller passes in.
+numbers itself -- it ranks by keys that the caller passes in; the correlation coefficient of a
+constant column (or of fewer than two samples) is NaN.
 """
 from __future__ import annotations
 
@@ -77,6 +78,8 @@ def pearson(length, sp, correct):
     cov = (x * y).sum() - sx * sy / n
     vx = (x * x).sum() - sx * sx / n
     vy = (y * y).sum() - sy * sy / n
+    if not vx * vy > 0:                                  # a constant column: the coefficient is undefined
+        return float("nan"), n
     return float(cov / np.sqrt(vx * vy)), n
 
 

@@ -38,6 +38,7 @@ EXPORTS = (
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
     "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade", "concur_prefill_attn",
+    "concur_curate",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -51,6 +52,22 @@ class concur_attn_config_t(ctypes.Structure):
         ("device", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
     ]
+
+
+class concur_curate_params_t(ctypes.Structure):
+    _fields_ = [
+        ("num_tasks", ctypes.c_int32), ("gens", ctypes.c_int32), ("rule_b_speedup", ctypes.c_float),
+        ("fast_p", ctypes.c_float), ("top_k", ctypes.c_int32), ("easy_below", ctypes.c_int32),
+        ("hard_above", ctypes.c_int32), ("reserved", ctypes.c_int32),
+    ]
+
+
+CONCUR_SEL_RANDOM, CONCUR_SEL_MAX_LENGTH, CONCUR_SEL_MIN_LENGTH, CONCUR_SEL_SPEEDUP = 0, 1, 2, 3
+(CONCUR_STAT_CORRECT, CONCUR_STAT_TASKS_CORRECT, CONCUR_STAT_RULE_A, CONCUR_STAT_RULE_B, CONCUR_STAT_LENGTH_SUM,
+ CONCUR_STAT_ARL, CONCUR_STAT_FAST_FIRST_COUNT, CONCUR_STAT_FAST_BEST_COUNT, CONCUR_STAT_EXEC_FIRST_COUNT,
+ CONCUR_STAT_N, CONCUR_STAT_SX, CONCUR_STAT_SY, CONCUR_STAT_SXX, CONCUR_STAT_SYY, CONCUR_STAT_SXY,
+ CONCUR_STAT_PEARSON_R, CONCUR_STAT_FAST_FIRST, CONCUR_STAT_FAST_BEST) = range(18)
+CONCUR_CURATE_NUM_STATS = 24
 
 
 def _load() -> ctypes.CDLL:
@@ -75,6 +92,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_decode_attn_cascade.restype = ctypes.c_int
     lib.concur_decode_attn_cascade.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp,
                                                i32, i32, i32, i32, vp]
+    lib.concur_curate.restype = ctypes.c_int
+    lib.concur_curate.argtypes = [ctypes.POINTER(concur_curate_params_t)] + [vp] * 14
     lib.concur_prefill_attn.restype = ctypes.c_int
     lib.concur_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_kv_append.restype = ctypes.c_int
@@ -196,6 +215,17 @@ def concur_prefill_attn(handle, q, k_pages, v_pages, block_table, seq_lens, q_st
                                  batch, total_q, num_pages, block_table_stride, stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_prefill_attn")
+    return rc
+
+
+def concur_curate(params: concur_curate_params_t, correct, t_torch, t_kernel, length, sample_key, task_key,
+                  speedup, rule_a, rule_b, pick, keep, difficulty, stats, stream=0, check=True) -> int:
+    """Curation arithmetic over [N][M] generation records (device tensors; see include/concur_curate.h)."""
+    rc = lib.concur_curate(ctypes.byref(params), _addr(correct), _addr(t_torch), _addr(t_kernel), _addr(length),
+                           _addr(sample_key), _addr(task_key), _addr(speedup), _addr(rule_a), _addr(rule_b),
+                           _addr(pick), _addr(keep), _addr(difficulty), _addr(stats), stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_curate")
     return rc
 
 

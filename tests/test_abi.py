@@ -1,5 +1,5 @@
 """The C-ABI shared library: it loads without a GPU, exports every function that
-include/concur_attn.h declares, and its host-only logic behaves."""
+include/*.h declares, and its host-only logic behaves."""
 import ctypes
 import re
 from pathlib import Path
@@ -19,9 +19,11 @@ def P():
 
 
 def declared_functions():
-    text = (ROOT / "include" / "concur_attn.h").read_text()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(concur_\w+)\s*\(", text)))
+    names = set()
+    for header in sorted((ROOT / "include").glob("*.h")):
+        text = re.sub(r"/\*.*?\*/", "", header.read_text(), flags=re.S)
+        names |= set(re.findall(r"\b(concur_\w+)\s*\(", text))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(P):

@@ -78,6 +78,7 @@ def test_pearson_closed_forms_and_library_special_case():
     assert abs(r - np.corrcoef(rec.length[m].astype(np.float64), sp[m].astype(np.float64))[0, 1]) < 1e-10
     mask = np.zeros_like(rec.correct); mask[0, 0] = 1
     assert np.isnan(C.pearson(rec.length, sp, mask)[0])              # fewer than two samples
+    assert np.isnan(C.pearson(np.full((10, 5), 7), sp[:10], ones)[0])    # a constant column
 
 
 def brute_rule_a(correct, sp, L):
