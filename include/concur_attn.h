@@ -87,7 +87,7 @@ typedef struct {
     int32_t num_q_heads;        /* Hq; supported: 8, 16, ... 64 (group size Hq/Hkv = 1 .. 8), e.g. 64 or 40 */
     int32_t num_kv_heads;       /* Hkv; supported: 8                                            */
     int32_t head_dim;           /* D; supported: 128                                            */
-    int32_t page_size;          /* P; supported: 16, 32, 64 tokens                              */
+    int32_t page_size;          /* P; supported: 16, 32, 64, 128 tokens                         */
     int32_t max_batch;          /* largest `batch` any call will pass (1 .. 65536)              */
     int32_t max_pages_per_seq;  /* largest `block_table_stride` any call will pass             */
     int32_t device;             /* CUDA device ordinal                                          */

@@ -40,7 +40,8 @@ int check_config(const concur_attn_config_t* c) {
     if (c->max_pages_per_seq < 1) return CONCUR_ERR_INVALID_ARG;
     if (c->num_kv_heads != kHkv || c->head_dim != kD) return CONCUR_ERR_UNSUPPORTED;
     if (c->num_q_heads < kHkv || c->num_q_heads > kHq || c->num_q_heads % kHkv != 0) return CONCUR_ERR_UNSUPPORTED;
-    if (c->page_size != 16 && c->page_size != 32 && c->page_size != 64) return CONCUR_ERR_UNSUPPORTED;
+    if (c->page_size != 16 && c->page_size != 32 && c->page_size != 64 && c->page_size != 128)
+        return CONCUR_ERR_UNSUPPORTED;
     // the flat tile index space must fit int32
     const int64_t tiles_per_seq = ((int64_t)c->max_pages_per_seq * c->page_size + kTile - 1) / kTile;
     if (tiles_per_seq * c->max_batch * kHkv >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
@@ -148,7 +149,9 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.num_pages = num_pages;
     p.bt_stride = stride;
     p.page_size = h->cfg.page_size;
-    p.page_shift = h->cfg.page_size == 16 ? 4 : (h->cfg.page_size == 32 ? 5 : 6);
+    p.page_shift = h->cfg.page_size == 16 ? 4 : (h->cfg.page_size == 32 ? 5 : (h->cfg.page_size == 64 ? 6 : 7));
+    p.box_rows = h->cfg.page_size < kTile ? h->cfg.page_size : kTile;
+    p.box_shift = p.page_shift < 6 ? p.page_shift : 6;
     p.hq = h->cfg.num_q_heads;
     p.group = h->cfg.num_q_heads / kHkv;
     const int per_sm = h->kernel == 1 ? partial_scalar_ctas_per_sm() : 1;
@@ -228,7 +231,7 @@ int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, voi
     DeviceGuard guard(h->cfg.device);
     if (!guard.ok()) return CONCUR_ERR_CUDA;
     const int32_t P = h->cfg.page_size;
-    const int32_t shift = P == 16 ? 4 : (P == 32 ? 5 : 6);
+    const int32_t shift = P == 16 ? 4 : (P == 32 ? 5 : (P == 64 ? 6 : 7));
     if (launch_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
                       reinterpret_cast<int32_t*>(h->ws + h->lay.hdr), batch, num_pages, block_table_stride, P,
                       shift, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)

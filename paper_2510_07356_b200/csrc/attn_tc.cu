@@ -95,7 +95,8 @@ struct TMeta {
     int32_t pages[4];     // physical pages of the tile (64 / P of them)
     int32_t nvalid;       // tokens of the tile that exist and that some row may see (1..64)
     int32_t diag;         // row group i sees columns c <= diag + i of the tile (>= 63: all of them)
-    int32_t pad[4];
+    int32_t row_in_page;  // first row of the tile inside its page (non-zero only for pages of more than 64 tokens)
+    int32_t pad[3];
 };
 static_assert(sizeof(TMeta) == 64, "one record per 64 bytes");
 
@@ -166,7 +167,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int32_t P = p.page_size;
+    const int32_t P = p.box_rows;            // rows per box: the unit of the shared-memory tile layout
 
     // unused query rows must at least be defined once
     for (int i = tid; i < (2 * kTQBytes) / 16; i += kTThreads)
@@ -204,8 +205,8 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         // =========================================================== producer warp
         uint32_t it = 0, vt = 0, seg = 0;                      // K tiles, V tiles, segments issued
         bool ok = true;
-        const int pages_per_tile_shift = 6 - p.page_shift;
-        const int32_t npages = kTile >> p.page_shift;
+        const int32_t npages = kTile >> p.box_shift;           // boxes per tile
+        const int32_t page_mask = p.page_size - 1;
         const uint32_t page_bytes = (uint32_t)P * 128u;        // one half of one page
         // V of tile u (lane 0 only): its pages are still in the tile's record
         auto issue_v = [&](uint32_t u) {
@@ -214,17 +215,17 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             ok = mbar_wait(empty_v(vs), ((u / kTVStages) & 1u) ^ 1u, abort_flag);
             if (!ok) return;
             const uint32_t vdst = smem_base + SM::kVOff + vs * kTTileBytes;
-            const int32_t npg = (m.nvalid + P - 1) >> p.page_shift;      // pages of the tile that are read
+            const int32_t npg = (m.nvalid + P - 1) >> p.box_shift;       // boxes of the tile that are read
             if (npages == 1) {
                 // page = tile: one box {64, 64, 2} lands as [half][row][128 B], the operand layout
                 mbar_arrive_expect_tx(full_v(vs), kTTileBytes);
-                tma_load_3d(vdst, &map_v, 0, (m.pages[0] * kHkv + m.g) * P, 0, full_v(vs));
+                tma_load_3d(vdst, &map_v, 0, (m.pages[0] * kHkv + m.g) * p.page_size + m.row_in_page, 0, full_v(vs));
             } else {
                 mbar_arrive_expect_tx(full_v(vs), npg * 2 * page_bytes);
                 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (q < npg) {
-                        const int32_t prow = (m.pages[q] * kHkv + m.g) * P;
+                        const int32_t prow = (m.pages[q] * kHkv + m.g) * p.page_size + m.row_in_page;
                         tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(vs));
                         tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(vs));
                     }
@@ -238,19 +239,20 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                                   int32_t row, int32_t qbase, int32_t pos0, int32_t pos_last) {
             const int32_t qsel = seg & 1;
             const int32_t tok_end = min(tile1 * kTile, pos_last + 1);
-            const int32_t page_end = (tok_end + P - 1) >> p.page_shift;
-            int32_t chunk_base = tile0 << pages_per_tile_shift;
+            const int32_t page_end = (tok_end + page_mask) >> p.page_shift;
+            int32_t chunk_base = (tile0 * kTile) >> p.page_shift;
             int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
             int32_t pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
             for (int32_t t = tile0; ok && t < tile1; ++t) {
-                const int32_t first_page = t << pages_per_tile_shift;
+                const int32_t first_page = (t * kTile) >> p.page_shift;
+                const int32_t row_in_page = (t * kTile) & page_mask;
                 if (first_page >= chunk_base + 32) {
                     chunk_base += 32;
                     pg = pg_next;
                     pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                 }
                 const int32_t nvalid = min(kTile, tok_end - t * kTile);
-                const int32_t npg = (nvalid + P - 1) >> p.page_shift;          // pages of the tile that are read
+                const int32_t npg = (nvalid + P - 1) >> p.box_shift;           // boxes of the tile that are read
                 const int ks = it % kTKStages;
                 int32_t my_page = __shfl_sync(0xffffffffu, pg, (first_page - chunk_base + (lane & 3)) & 31);
                 const bool bad = (lane < npg) && (my_page < 0 || my_page >= p.num_pages);
@@ -279,19 +281,19 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                         TMeta& m = meta[it % kTMetaRing];
                         m.n = n; m.idx = t - tile0; m.cnt = tile1 - tile0; m.qsel = qsel; m.row = row; m.g = g;
                         m.pages[0] = pages[0]; m.pages[1] = pages[1]; m.pages[2] = pages[2]; m.pages[3] = pages[3];
-                        m.nvalid = nvalid;
+                        m.nvalid = nvalid; m.row_in_page = row_in_page;
                         m.diag = kPrefill ? min(pos0 - t * kTile, 1 << 20) : (1 << 20);
                         mbar_arrive(meta_full(it % kTMetaRing));
                         const uint32_t kdst = smem_base + ks * kTTileBytes;
                         if (npages == 1) {
                             mbar_arrive_expect_tx(full_k(ks), kTTileBytes);
-                            tma_load_3d(kdst, &map_k, 0, (pages[0] * kHkv + g) * P, 0, full_k(ks));
+                            tma_load_3d(kdst, &map_k, 0, (pages[0] * kHkv + g) * p.page_size + row_in_page, 0, full_k(ks));
                         } else {
                             mbar_arrive_expect_tx(full_k(ks), npg * 2 * page_bytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
                                 if (q < npg) {
-                                    const int32_t prow = (pages[q] * kHkv + g) * P;
+                                    const int32_t prow = (pages[q] * kHkv + g) * p.page_size + row_in_page;
                                     tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
                                     tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
                                 }
@@ -334,7 +336,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         } else {
             // prefill: unit r = (sequence b, block of 16 query tokens, KV head g); the blocks of a
             // sequence are taken last first (they have the most tiles); a unit is never split
-            const int64_t max_len = (int64_t)p.bt_stride * P;
+            const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
             while (ok && r < W) {
                 int32_t r_next = 0;
                 if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
@@ -737,9 +739,9 @@ cudaError_t launch_attn_tc(const DecodeParams& p, const CascadeParams& c, const 
     CUtensorMap mk, mv, mq;
     const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
     // a 64-token page is a whole tile: both halves come with one copy ([half][row][128 B])
-    const uint32_t halves = p.page_size == kTile ? 2 : 1;
-    if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.page_size, halves) ||
-        !make_half_row_map(&mv, p.v_pages, pool_rows, p.page_size, halves) ||
+    const uint32_t halves = p.box_rows == kTile ? 2 : 1;
+    if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.box_rows, halves) ||
+        !make_half_row_map(&mv, p.v_pages, pool_rows, p.box_rows, halves) ||
         !make_half_row_map(&mq, p.q, q_rows, kGroup))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<kPrefill>, cudaFuncAttributeMaxDynamicSharedMemorySize,

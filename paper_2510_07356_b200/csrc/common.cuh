@@ -44,6 +44,8 @@ struct DecodeParams {
     int32_t bt_stride;
     int32_t page_size;
     int32_t page_shift;       // log2(page_size)
+    int32_t box_rows;         // rows of one TMA box = min(page_size, 64): a 64-token tile is 64 / box_rows boxes
+    int32_t box_shift;        // log2(box_rows)
     int32_t group;            // query heads per KV head (1..kGroup); heads g*group .. g*group+group-1 share KV head g
     int32_t hq;               // query heads = kHkv * group
     // plan controls

@@ -105,8 +105,8 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int32_t P = p.page_size;
-    const int64_t max_len = (int64_t)p.bt_stride * P;
+    const int32_t P = p.box_rows;            // rows per box: the unit of the shared-memory tile layout
+    const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
     const bool cached = p.batch <= kSmemBatch;
 
     if (tid == 0) {
@@ -150,8 +150,8 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         uint32_t it = 0;                       // tiles issued so far
         int32_t r = blockIdx.x;                // CTA i starts on range i; further ranges are claimed
         bool ok = true;
-        const int pages_per_tile_shift = 6 - p.page_shift;      // log2(64 / P)
         const uint32_t box_bytes = (uint32_t)P * kRowBytes;
+        const int32_t page_mask = p.page_size - 1;
         while (ok && r < R) {
             // the next range is claimed a few tiles before this one ends: late enough that no
             // CTA sits on work another could start, early enough to hide the atomic's latency
@@ -169,10 +169,10 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 // cascade mode: the first `off` tokens (a multiple of 64) belong to the prefix pass
                 const int32_t off = p.tok_offset ? p.tok_offset[sg.b] : 0;
                 n -= off;
-                const int32_t page_off = off >> p.page_shift;
                 const int32_t* table = p.block_table + (int64_t)sg.b * p.bt_stride;
-                const int32_t page_end = page_off + ((min(sg.tile1 * kTile, n) + P - 1) >> p.page_shift);   // pages used by the segment
-                int32_t chunk_base = page_off + (sg.tile0 << pages_per_tile_shift);
+                // pages used by the segment (a page holds one or more boxes; a 128-token page two tiles)
+                const int32_t page_end = (off + min(sg.tile1 * kTile, n) + page_mask) >> p.page_shift;
+                int32_t chunk_base = (off + sg.tile0 * kTile) >> p.page_shift;
                 // this lane's entry of the current 32-page chunk of the block table, and of the
                 // chunk after it (fetched one chunk early so that its latency never stalls the ring)
                 int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
@@ -183,14 +183,16 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                         if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
                         claimed = true;
                     }
-                    const int32_t first_page = page_off + (t << pages_per_tile_shift);
+                    const int32_t tok_abs = off + t * kTile;               // first token of the tile in its sequence
+                    const int32_t first_page = tok_abs >> p.page_shift;
+                    const int32_t row_in_page = tok_abs & page_mask;       // non-zero only for pages of more than 64 tokens
                     if (first_page >= chunk_base + 32) {
                         chunk_base += 32;
                         pg = pg_next;
                         pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                     }
                     const int32_t n_valid = min(kTile, n - t * kTile);
-                    const int32_t npages = (n_valid + P - 1) >> p.page_shift;
+                    const int32_t npages = (n_valid + P - 1) >> p.box_shift;      // boxes of the tile that are read
                     const int s = it % kStages;
                     const uint32_t parity = (it / kStages) & 1u;
                     // page ids of this tile, clamped into the pool
@@ -223,12 +225,12 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                             #pragma unroll
                             for (int i = 0; i < 4; ++i)
                                 if (i < npages)
-                                    tma_load_tile(kdst + i * box_bytes, &map_k, (pages[i] * kHkv + sg.g) * P, full_k(s));
+                                    tma_load_tile(kdst + i * box_bytes, &map_k, (pages[i] * kHkv + sg.g) * p.page_size + row_in_page, full_k(s));
                             mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
                             #pragma unroll
                             for (int i = 0; i < 4; ++i)
                                 if (i < npages)
-                                    tma_load_tile(vdst + i * box_bytes, &map_v, (pages[i] * kHkv + sg.g) * P, full_v(s));
+                                    tma_load_tile(vdst + i * box_bytes, &map_v, (pages[i] * kHkv + sg.g) * p.page_size + row_in_page, full_v(s));
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -339,7 +341,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     // a 64-token tile is 64/P boxes; a box is [2 halves][P rows][128 B], 16-byte chunks of a
     // row XOR-ed with (row & 7)
     const int tok0 = warp * 16;                                   // this warp's first token in the tile
-    const uint32_t box_off = (uint32_t)(tok0 >> p.page_shift) * (uint32_t)P * kRowBytes;
+    const uint32_t box_off = (uint32_t)(tok0 >> p.box_shift) * (uint32_t)P * kRowBytes;
     const uint32_t half_stride = (uint32_t)P * 128u;
     const int rb0 = tok0 & (P - 1);
     // K fragments (non-transposed): matrices (rows 0-7 | 8-15) x (k 0-7 | 8-15)
@@ -567,7 +569,7 @@ bool make_pool_map(CUtensorMap* map, const void* pool, int32_t num_pages, int32_
     if (!fn) return false;
     const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * kHkv * P, 2};
     const cuuint64_t strides[2] = {256, 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)P, 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)(P < kTile ? P : kTile), 2};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pool), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -82,7 +82,7 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int32_t P = p.page_size;
+    const int32_t P = p.box_rows;            // rows per box: the unit of the shared-memory tile layout
 
     if (tid == 0) {
         for (int s = 0; s < kPStages; ++s) {
@@ -105,8 +105,8 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
         // =========================================================== producer warp
         uint32_t it = 0, seg = 0;
         bool ok = true;
-        const int pages_per_tile_shift = 6 - p.page_shift;
         const uint32_t box_bytes = (uint32_t)P * kRowBytes;
+        const int32_t page_mask = p.page_size - 1;
         int32_t r = blockIdx.x;
         while (ok && r < R) {
             int32_t r_next = 0;
@@ -129,18 +129,19 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                 const int32_t row = c.unit_rowbase[i * kHkv + g] + split * n;
                 const int32_t qsel = seg & 1;
                 const int32_t* table = p.block_table + (int64_t)b0 * p.bt_stride;   // the first sibling's pages
-                const int32_t page_end = tile1 << pages_per_tile_shift;
-                int32_t chunk_base = tile0 << pages_per_tile_shift;
+                const int32_t page_end = (tile1 * kTile + page_mask) >> p.page_shift;
+                int32_t chunk_base = (tile0 * kTile) >> p.page_shift;
                 int32_t pg = (chunk_base + lane < page_end) ? __ldg(table + chunk_base + lane) : 0;
                 int32_t pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                 for (int32_t t = tile0; ok && t < tile1; ++t) {
-                    const int32_t first_page = t << pages_per_tile_shift;
+                    const int32_t first_page = (t * kTile) >> p.page_shift;
+                    const int32_t row_in_page = (t * kTile) & page_mask;   // non-zero only for pages of more than 64 tokens
                     if (first_page >= chunk_base + 32) {
                         chunk_base += 32;
                         pg = pg_next;
                         pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                     }
-                    const int32_t npages = kTile >> p.page_shift;
+                    const int32_t npages = kTile >> p.box_shift;          // boxes per tile
                     const int s = it % kPStages;
                     const uint32_t parity = (it / kPStages) & 1u;
                     int32_t my_page = __shfl_sync(0xffffffffu, pg, (first_page - chunk_base + (lane & 3)) & 31);
@@ -171,11 +172,11 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                             mbar_arrive_expect_tx(full_k(s), npages * box_bytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
-                                if (q < npages) tma_load_tile(kdst + q * box_bytes, &map_k, (pages[q] * kHkv + g) * P, full_k(s));
+                                if (q < npages) tma_load_tile(kdst + q * box_bytes, &map_k, (pages[q] * kHkv + g) * p.page_size + row_in_page, full_k(s));
                             mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
-                                if (q < npages) tma_load_tile(vdst + q * box_bytes, &map_v, (pages[q] * kHkv + g) * P, full_v(s));
+                                if (q < npages) tma_load_tile(vdst + q * box_bytes, &map_v, (pages[q] * kHkv + g) * p.page_size + row_in_page, full_v(s));
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -210,7 +211,7 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
     const int tok0 = warp * 16;
     const uint32_t half_stride = (uint32_t)P * 128u;
     // K fragments of this warp's 16 tokens (phase 1)
-    const uint32_t k_box_off = (uint32_t)(tok0 >> p.page_shift) * (uint32_t)P * kRowBytes;
+    const uint32_t k_box_off = (uint32_t)(tok0 >> p.box_shift) * (uint32_t)P * kRowBytes;
     const int k_row = (tok0 & (P - 1)) + (lane & 7) + ((lane >> 3) & 1) * 8;
     const uint32_t k_row_off = k_box_off + (uint32_t)k_row * 128u;
     const int k_sel = lane >> 4;
@@ -335,7 +336,7 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                     const int tok = (2 * tp + tb) * 16 + (lane & 7) + (lane >> 4) * 8;
                     const int chunk = (2 * warp + db) * 2 + ((lane >> 3) & 1);
                     const int rb = tok & (P - 1);
-                    const uint32_t addr = vbase + (uint32_t)(tok >> p.page_shift) * (uint32_t)P * kRowBytes +
+                    const uint32_t addr = vbase + (uint32_t)(tok >> p.box_shift) * (uint32_t)P * kRowBytes +
                                           (uint32_t)(chunk >> 3) * half_stride + (uint32_t)rb * 128u +
                                           (uint32_t)(((chunk & 7) ^ (rb & 7)) << 4);
                     ldmatrix_x4_trans(addr, va[db][tb]);
@@ -459,7 +460,7 @@ cudaError_t launch_ns(const DecodeParams& p, const CascadeParams& c, const CUten
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
     const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
-    if (!make_row_map(&mk, p.k_pages, pool_rows, p.page_size) || !make_row_map(&mv, p.v_pages, pool_rows, p.page_size) ||
+    if (!make_row_map(&mk, p.k_pages, pool_rows, p.box_rows) || !make_row_map(&mv, p.v_pages, pool_rows, p.box_rows) ||
         !make_row_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup))
         return cudaErrorInvalidValue;
     return launch_ns<kMaxShare>(p, c, mk, mv, mq, stream);

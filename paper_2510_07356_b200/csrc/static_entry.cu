@@ -104,6 +104,8 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.bt_stride = block_table_stride;
     p.page_size = page_size;
     p.page_shift = page_size == 16 ? 4 : (page_size == 32 ? 5 : 6);
+    p.box_rows = page_size;
+    p.box_shift = p.page_shift;
     p.hq = kHq;
     p.group = kGroup;
     p.grid_ctas = s->sm_count;

@@ -46,12 +46,13 @@ GROUPS = [
 ]
 
 
-@pytest.mark.parametrize("page_size", [16, 32, 64])
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128])
 @pytest.mark.parametrize("kernel", [0, 1])
 @pytest.mark.parametrize("prefix_kernel", [0, 1])
 def test_cascade_matches_oracle(P, page_size, kernel, prefix_kernel):
     """prefix_kernel 0: tcgen05 / TMEM prefix pass; 1: warp-level mma.sync prefix pass."""
-    cw = synth.make_cascade_workload(f"casc_p{page_size}", GROUPS, page_size, 4000 + page_size, "cuda:0")
+    groups = [(shared - shared % page_size, owns) for shared, owns in GROUPS]      # only whole pages can be shared
+    cw = synth.make_cascade_workload(f"casc_p{page_size}", groups, page_size, 4000 + page_size, "cuda:0")
     out, lse, attn = run_cascade(P, cw, kernel=kernel, prefix_kernel=prefix_kernel)
     assert attn.status() == 0
     ref_out, ref_lse = oracle_sequences(synth.gather_sequences(cw.w, range(cw.w.spec.batch)))

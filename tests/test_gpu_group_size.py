@@ -27,7 +27,7 @@ def host(w):
 
 @pytest.mark.parametrize("hq", [8, 16, 24, 40, 56])
 @pytest.mark.parametrize("kernel", [0, 1])
-@pytest.mark.parametrize("page_size,ranges", [(16, 0), (64, 0), (64, 7), (32, 300)])
+@pytest.mark.parametrize("page_size,ranges", [(16, 0), (64, 0), (64, 7), (32, 300), (128, 0), (128, 9)])
 def test_plain_step_with_smaller_groups(P, hq, kernel, page_size, ranges):
     spec = synth.tiny_spec(f"g{hq}", LENS, page_size, 7000 + hq, num_q_heads=hq)
     w = synth.make_workload(spec, "cuda:0")

@@ -39,7 +39,7 @@ EDGE_LENS = (0, 1, 2, 15, 16, 17, 31, 33, 63, 64, 65, 127, 128, 129, 191, 200, 2
 
 
 @pytest.mark.parametrize("kernel", list(KERNELS))
-@pytest.mark.parametrize("page_size", [16, 32, 64])
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128])
 @pytest.mark.parametrize("ranges", [0, 1, 2, 3, 7, 61, 4736])
 def test_edge_lengths_and_forced_splits(P, kernel, page_size, ranges):
     spec = synth.tiny_spec(f"edge_p{page_size}", EDGE_LENS, page_size, 1000 + page_size)

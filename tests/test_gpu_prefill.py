@@ -48,13 +48,13 @@ def check(P, pw, tokens=None, hq=64, what=""):
 LENS = (1, 2, 15, 16, 17, 63, 64, 65, 100, 129, 200, 333)
 
 
-@pytest.mark.parametrize("page_size", [64, 16, 32])
+@pytest.mark.parametrize("page_size", [64, 16, 32, 128])
 def test_whole_prompts_every_token(P, page_size):
     pw = synth.make_prefill_workload(f"pf_p{page_size}", LENS, LENS, page_size, 9000 + page_size, "cuda:0")
     check(P, pw, what=f"whole prompts p{page_size}")
 
 
-@pytest.mark.parametrize("page_size", [16, 64])
+@pytest.mark.parametrize("page_size", [16, 64, 128])
 def test_chunks_at_the_end_of_longer_contexts(P, page_size):
     lens = (500, 64, 1000, 129, 2049, 77, 640)
     q_lens = (1, 64, 17, 100, 48, 0, 333)           # one sequence has no query token at all

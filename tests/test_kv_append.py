@@ -90,7 +90,7 @@ def _check_step(final, lens_now, q, out, lse, what):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("page_size", [16, 64])
+@pytest.mark.parametrize("page_size", [16, 64, 128])
 def test_append_then_attend_loop(P, page_size):
     lens0, steps = [100, 63, 0, 1000, 15], 5
     final, k, v, k_new, v_new, q_steps = _loop_case(page_size, lens0, steps, 900 + page_size)
