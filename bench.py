@@ -59,6 +59,7 @@ def parse_args():
     ap.add_argument("--loop-steps", type=int, default=16, help="append+attention steps replayed from a CUDA graph")
     ap.add_argument("--fuse-combine", type=int, default=-1)
     ap.add_argument("--claim-ahead", type=int, default=-1)
+    ap.add_argument("--kv-layout", type=int, default=0, help="decode workloads: 0 head-major pools, 1 token-major")
     ap.add_argument("--prefix-kernel", type=int, default=0, help="cascade workloads: 0 tcgen05 prefix pass, 1 mma.sync")
     return ap.parse_args()
 
@@ -604,7 +605,11 @@ def main():
     spec = rank_spec(synth.SPECS[args.workload], rank, world)
     w = synth.make_workload(spec, dev, spare_tokens=args.loop_steps)
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local,
-                             num_q_heads=spec.num_q_heads)
+                             num_q_heads=spec.num_q_heads, kv_layout=args.kv_layout)
+    if args.kv_layout == 1:              # the same cache as [page][slot][KV head][D]
+        w.k_pages = w.k_pages.permute(0, 2, 1, 3).contiguous()
+        w.v_pages = w.v_pages.permute(0, 2, 1, 3).contiguous()
+        args.no_cpu = True               # the oracle reads head-major pools; parity is the tests' business
     attn.set_option(P.CONCUR_OPT_KERNEL, args.kernel)
     attn.set_option(P.CONCUR_OPT_RANGES_PER_CTA, args.ranges_per_cta)
     attn.set_option(P.CONCUR_OPT_MIN_RANGE_TILES, args.min_range_tiles)
@@ -764,6 +769,7 @@ def main():
                    "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128, "algorithmic_bytes": nbytes,
                    "l2": "flushed between steps" if flush_needed else "inputs larger than L2",
                    "kernel": "mma" if args.kernel == 0 else "scalar", "ranges": R, "tiles": W,
+                   "kv_layout": "token-major" if args.kv_layout == 1 else "head-major",
                    "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
         "kv_tokens_per_s": job_tokens / (ms_per_step * 1e-3),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,

@@ -24,7 +24,8 @@
  *
  * Memory layout (all device memory unless a parameter says otherwise; caller-owned):
  *     q            bf16  [batch][Hq][D]
- *     k_pages      bf16  [num_pages][Hkv][P][D]        one (page, head) tile is contiguous
+ *     k_pages      bf16  [num_pages][Hkv][P][D]        one (page, head) tile is contiguous; or, with
+ *                        kv_layout = CONCUR_KV_TOKEN_MAJOR, [num_pages][P][Hkv][D]
  *     v_pages      bf16  same shape; K and V of a token share page id and slot
  *     block_table  int32 [batch][block_table_stride]   logical page i of b -> physical page
  *     seq_lens     int32 [batch]
@@ -81,6 +82,10 @@ typedef enum {
 #define CONCUR_OPT_PREFIX_KERNEL 10 /* shared-prefix pass of the cascade step: 0 (default) = tcgen05 kernel with
                                        TMEM accumulators, 1 = warp-level mma.sync kernel                 */
 
+/* Layouts of the K and V pools (concur_attn_config_t.kv_layout). */
+#define CONCUR_KV_HEAD_MAJOR  0   /* [num_pages][Hkv][P][D]: one (page, head) tile is contiguous (default) */
+#define CONCUR_KV_TOKEN_MAJOR 1   /* [num_pages][P][Hkv][D]: one token's rows of all KV heads are contiguous */
+
 typedef struct concur_attn concur_attn_t;   /* opaque; owns its workspace and nothing else */
 
 typedef struct {
@@ -91,7 +96,7 @@ typedef struct {
     int32_t max_batch;          /* largest `batch` any call will pass (1 .. 65536)              */
     int32_t max_pages_per_seq;  /* largest `block_table_stride` any call will pass             */
     int32_t device;             /* CUDA device ordinal                                          */
-    int32_t reserved;           /* must be 0                                                    */
+    int32_t kv_layout;          /* CONCUR_KV_HEAD_MAJOR (0, default) or CONCUR_KV_TOKEN_MAJOR   */
     void*   workspace;          /* optional device memory (256-byte aligned) of at least
                                    concur_attn_workspace_bytes(); NULL: the library allocates  */
     size_t  workspace_bytes;    /* size of `workspace`; ignored when it is NULL                */

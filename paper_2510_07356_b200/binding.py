@@ -22,6 +22,9 @@ CONCUR_FLAG_BAD_PAGE_ID = 1
 CONCUR_FLAG_BAD_SEQ_LEN = 2
 CONCUR_FLAG_WAIT_LIMIT = 4
 
+CONCUR_KV_HEAD_MAJOR = 0
+CONCUR_KV_TOKEN_MAJOR = 1
+
 CONCUR_OPT_KERNEL = 1
 CONCUR_OPT_NUM_RANGES = 2
 CONCUR_OPT_GRID_CTAS = 3
@@ -49,7 +52,7 @@ class concur_attn_config_t(ctypes.Structure):
         ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
         ("max_batch", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
-        ("device", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("device", ctypes.c_int32), ("kv_layout", ctypes.c_int32),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
     ]
 
@@ -126,9 +129,9 @@ def concur_attn_strerror(code: int) -> str:
 
 def make_config(page_size: int, max_batch: int, max_pages_per_seq: int, device: int = 0,
                 num_q_heads: int = 64, num_kv_heads: int = 8, head_dim: int = 128,
-                workspace: int = 0, workspace_bytes: int = 0) -> concur_attn_config_t:
+                workspace: int = 0, workspace_bytes: int = 0, kv_layout: int = 0) -> concur_attn_config_t:
     return concur_attn_config_t(num_q_heads, num_kv_heads, head_dim, page_size, max_batch,
-                                max_pages_per_seq, device, 0, workspace or None, workspace_bytes)
+                                max_pages_per_seq, device, kv_layout, workspace or None, workspace_bytes)
 
 
 def concur_attn_workspace_bytes(cfg: concur_attn_config_t) -> int:

@@ -35,7 +35,8 @@ WorkspaceLayout layout_for(int32_t max_batch) {
 
 int check_config(const concur_attn_config_t* c) {
     if (!c) return CONCUR_ERR_INVALID_ARG;
-    if (c->reserved != 0 || c->device < 0) return CONCUR_ERR_INVALID_ARG;
+    if ((c->kv_layout != CONCUR_KV_HEAD_MAJOR && c->kv_layout != CONCUR_KV_TOKEN_MAJOR) || c->device < 0)
+        return CONCUR_ERR_INVALID_ARG;
     if (c->max_batch < 1 || c->max_batch > kMaxBatchLimit) return CONCUR_ERR_INVALID_ARG;
     if (c->max_pages_per_seq < 1) return CONCUR_ERR_INVALID_ARG;
     if (c->num_kv_heads != kHkv || c->head_dim != kD) return CONCUR_ERR_UNSUPPORTED;
@@ -152,6 +153,7 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.page_shift = h->cfg.page_size == 16 ? 4 : (h->cfg.page_size == 32 ? 5 : (h->cfg.page_size == 64 ? 6 : 7));
     p.box_rows = h->cfg.page_size < kTile ? h->cfg.page_size : kTile;
     p.box_shift = p.page_shift < 6 ? p.page_shift : 6;
+    p.token_major = h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0;
     p.hq = h->cfg.num_q_heads;
     p.group = h->cfg.num_q_heads / kHkv;
     const int per_sm = h->kernel == 1 ? partial_scalar_ctas_per_sm() : 1;
@@ -234,7 +236,8 @@ int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, voi
     const int32_t shift = P == 16 ? 4 : (P == 32 ? 5 : (P == 64 ? 6 : 7));
     if (launch_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
                       reinterpret_cast<int32_t*>(h->ws + h->lay.hdr), batch, num_pages, block_table_stride, P,
-                      shift, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+                      shift, h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0,
+                      static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return CONCUR_ERR_CUDA;
     return CONCUR_OK;
 }

@@ -219,15 +219,15 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             if (npages == 1) {
                 // page = tile: one box {64, 64, 2} lands as [half][row][128 B], the operand layout
                 mbar_arrive_expect_tx(full_v(vs), kTTileBytes);
-                tma_load_3d(vdst, &map_v, 0, (m.pages[0] * kHkv + m.g) * p.page_size + m.row_in_page, 0, full_v(vs));
+                tma_load_3d(vdst, &map_v, 0, pool_row(p, m.pages[0], m.g, m.row_in_page), pool_plane(p, m.g), full_v(vs));
             } else {
                 mbar_arrive_expect_tx(full_v(vs), npg * 2 * page_bytes);
                 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (q < npg) {
-                        const int32_t prow = (m.pages[q] * kHkv + m.g) * p.page_size + m.row_in_page;
-                        tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, 0, full_v(vs));
-                        tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, 1, full_v(vs));
+                        const int32_t prow = pool_row(p, m.pages[q], m.g, m.row_in_page), pl = pool_plane(p, m.g);
+                        tma_load_3d(vdst + q * page_bytes, &map_v, 0, prow, pl, full_v(vs));
+                        tma_load_3d(vdst + kTHalfBytes + q * page_bytes, &map_v, 0, prow, pl + 1, full_v(vs));
                     }
             }
             ++vt;
@@ -287,15 +287,15 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                         const uint32_t kdst = smem_base + ks * kTTileBytes;
                         if (npages == 1) {
                             mbar_arrive_expect_tx(full_k(ks), kTTileBytes);
-                            tma_load_3d(kdst, &map_k, 0, (pages[0] * kHkv + g) * p.page_size + row_in_page, 0, full_k(ks));
+                            tma_load_3d(kdst, &map_k, 0, pool_row(p, pages[0], g, row_in_page), pool_plane(p, g), full_k(ks));
                         } else {
                             mbar_arrive_expect_tx(full_k(ks), npg * 2 * page_bytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
                                 if (q < npg) {
-                                    const int32_t prow = (pages[q] * kHkv + g) * p.page_size + row_in_page;
-                                    tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, 0, full_k(ks));
-                                    tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, 1, full_k(ks));
+                                    const int32_t prow = pool_row(p, pages[q], g, row_in_page), pl = pool_plane(p, g);
+                                    tma_load_3d(kdst + q * page_bytes, &map_k, 0, prow, pl, full_k(ks));
+                                    tma_load_3d(kdst + kTHalfBytes + q * page_bytes, &map_k, 0, prow, pl + 1, full_k(ks));
                                 }
                         }
                         if (it >= (uint32_t)kTVLag) issue_v(it - kTVLag);
@@ -721,11 +721,13 @@ EncodeTiledFn encode_fn() {
 // Rows of 128 bf16 seen as {64 elements, rows, 2 halves}; a box is `box_rows` rows of ONE half
 // and lands in shared memory as [row][128 B] with the 128-byte swizzle: one slab of a K-major
 // (or, read along the rows, MN-major) tcgen05 operand.
-bool make_half_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, uint32_t box_halves = 1) {
+bool make_half_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, uint32_t box_halves = 1,
+                       int planes = 2) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {64, rows, 2};
-    const cuuint64_t strides[2] = {256, 128};
+    // planes = 2: rows of 128 elements; planes = 16: token-major pool rows (8 heads x 2 halves per token)
+    const cuuint64_t dims[3] = {64, rows, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)planes * 128, 128};
     const cuuint32_t box[3] = {64, box_rows, box_halves};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -737,11 +739,12 @@ template <bool kPrefill>
 cudaError_t launch_attn_tc(const DecodeParams& p, const CascadeParams& c, const PrefillParams& f, uint64_t q_rows,
                            int grid, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
-    const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
+    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
+    const int planes = p.token_major ? 2 * kHkv : 2;
     // a 64-token page is a whole tile: both halves come with one copy ([half][row][128 B])
     const uint32_t halves = p.box_rows == kTile ? 2 : 1;
-    if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.box_rows, halves) ||
-        !make_half_row_map(&mv, p.v_pages, pool_rows, p.box_rows, halves) ||
+    if (!make_half_row_map(&mk, p.k_pages, pool_rows, p.box_rows, halves, planes) ||
+        !make_half_row_map(&mv, p.v_pages, pool_rows, p.box_rows, halves, planes) ||
         !make_half_row_map(&mq, p.q, q_rows, kGroup))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<kPrefill>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -46,6 +46,7 @@ struct DecodeParams {
     int32_t page_shift;       // log2(page_size)
     int32_t box_rows;         // rows of one TMA box = min(page_size, 64): a 64-token tile is 64 / box_rows boxes
     int32_t box_shift;        // log2(box_rows)
+    int32_t token_major;      // 0: pools are [page][KV head][slot][D]; 1: [page][slot][KV head][D]
     int32_t group;            // query heads per KV head (1..kGroup); heads g*group .. g*group+group-1 share KV head g
     int32_t hq;               // query heads = kHkv * group
     // plan controls
@@ -92,6 +93,18 @@ struct PrefillParams {
     const int32_t* q_start;       // [batch + 1] first query token of each sequence in q / out; last entry = total_q
     int32_t total_q;
 };
+
+// Where token `slot` of KV head g of page `page` sits, as the (row, half-plane) coordinates of the
+// tensor maps over a pool (a row is 64 elements of one half of one 128-wide K or V row; `half` is
+// added to the plane by the caller) and as an element offset for plain loads and stores.
+__device__ __forceinline__ int32_t pool_row(const DecodeParams& p, int32_t page, int32_t g, int32_t slot) {
+    return p.token_major ? page * p.page_size + slot : (page * kHkv + g) * p.page_size + slot;
+}
+__device__ __forceinline__ int32_t pool_plane(const DecodeParams& p, int32_t g) { return p.token_major ? 2 * g : 0; }
+__device__ __forceinline__ int64_t pool_elem(const DecodeParams& p, int32_t page, int32_t g, int32_t slot) {
+    return p.token_major ? (((int64_t)page * p.page_size + slot) * kHkv + g) * kD
+                         : (((int64_t)page * kHkv + g) * p.page_size + slot) * kD;
+}
 
 // First flat tile of range r when [0, W) is cut into R ranges of equal size.
 __device__ __forceinline__ int32_t range_begin(int32_t W, int32_t R, int32_t r) {
@@ -171,6 +184,6 @@ int partial_scalar_ctas_per_sm();
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                           const int32_t* block_table, int32_t* seq_lens, int32_t* hdr, int32_t batch,
                           int32_t num_pages, int32_t bt_stride, int32_t page_size, int32_t page_shift,
-                          cudaStream_t stream);
+                          int32_t token_major, cudaStream_t stream);
 
 }  // namespace concur

@@ -225,12 +225,12 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                             #pragma unroll
                             for (int i = 0; i < 4; ++i)
                                 if (i < npages)
-                                    tma_load_tile(kdst + i * box_bytes, &map_k, (pages[i] * kHkv + sg.g) * p.page_size + row_in_page, full_k(s));
+                                    tma_load_tile(kdst + i * box_bytes, &map_k, pool_row(p, pages[i], sg.g, row_in_page), full_k(s), pool_plane(p, sg.g));
                             mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
                             #pragma unroll
                             for (int i = 0; i < 4; ++i)
                                 if (i < npages)
-                                    tma_load_tile(vdst + i * box_bytes, &map_v, (pages[i] * kHkv + sg.g) * p.page_size + row_in_page, full_v(s));
+                                    tma_load_tile(vdst + i * box_bytes, &map_v, pool_row(p, pages[i], sg.g, row_in_page), full_v(s), pool_plane(p, sg.g));
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -564,11 +564,14 @@ EncodeTiledFn encode_fn() {
 // A pool [num_pages][8][P][128] bf16 seen as {64 elements, rows, 2 halves}: element stride 2 B,
 // row stride 256 B, half stride 128 B.  A box {64, P, 2} is one (page, head) chunk and lands in
 // shared memory as [half][row][128 B] with the 128-byte swizzle.
-bool make_pool_map(CUtensorMap* map, const void* pool, int32_t num_pages, int32_t P) {
+bool make_pool_map(CUtensorMap* map, const void* pool, int32_t num_pages, int32_t P, int32_t token_major) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * kHkv * P, 2};
-    const cuuint64_t strides[2] = {256, 128};
+    // token-major pools [page][slot][8][128]: a row (token) is 2 KB apart and the 16 half-planes of
+    // its 8 heads are 128 B apart; the box is the same {64, rows, 2}, at plane 2 g
+    const cuuint64_t dims[3] = {64, token_major ? (cuuint64_t)num_pages * P : (cuuint64_t)num_pages * kHkv * P,
+                                token_major ? (cuuint64_t)(2 * kHkv) : 2};
+    const cuuint64_t strides[2] = {token_major ? (cuuint64_t)(kHkv * 256) : 256, 128};
     const cuuint32_t box[3] = {64, (cuuint32_t)(P < kTile ? P : kTile), 2};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pool), dims, strides, box, estr,
@@ -592,8 +595,8 @@ cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
         if (e != cudaSuccess) return e;
     }
     CUtensorMap map_k, map_v;
-    if (!make_pool_map(&map_k, p.k_pages, p.num_pages, p.page_size) ||
-        !make_pool_map(&map_v, p.v_pages, p.num_pages, p.page_size))
+    if (!make_pool_map(&map_k, p.k_pages, p.num_pages, p.page_size, p.token_major) ||
+        !make_pool_map(&map_v, p.v_pages, p.num_pages, p.page_size, p.token_major))
         return cudaErrorInvalidValue;
     // programmatic dependent launch: the prologue (barrier set-up) may overlap the plan kernel
     cudaLaunchConfig_t cfg = {};

@@ -88,16 +88,17 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
                     if (sub == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagBadPage);
                 }
                 const int32_t slot = t & (p.page_size - 1);
-                const int64_t row = ((int64_t)page * kHkv + sg.g) * p.page_size + slot;
-                const uint4* kp = reinterpret_cast<const uint4*>(p.k_pages + row * kD) + sub;
-                const uint4* vp = reinterpret_cast<const uint4*>(p.v_pages + row * kD) + sub;
+                const int64_t elem = pool_elem(p, page, sg.g, slot);
+                const int64_t tok_stride = p.token_major ? kHkv * (kD / 8) : kD / 8;   // uint4s between consecutive tokens
+                const uint4* kp = reinterpret_cast<const uint4*>(p.k_pages + elem) + sub;
+                const uint4* vp = reinterpret_cast<const uint4*>(p.v_pages + elem) + sub;
                 uint4 kr[kTokPerStep], vr[kTokPerStep];
                 bool valid[kTokPerStep];
                 #pragma unroll
                 for (int i = 0; i < kTokPerStep; ++i) {
                     valid[i] = (t + i) < tok1;
-                    kr[i] = valid[i] ? __ldg(kp + i * (kD / 8)) : make_uint4(0, 0, 0, 0);
-                    vr[i] = valid[i] ? __ldg(vp + i * (kD / 8)) : make_uint4(0, 0, 0, 0);
+                    kr[i] = valid[i] ? __ldg(kp + i * tok_stride) : make_uint4(0, 0, 0, 0);
+                    vr[i] = valid[i] ? __ldg(vp + i * tok_stride) : make_uint4(0, 0, 0, 0);
                 }
                 float s[kTokPerStep][kGroup];
                 #pragma unroll

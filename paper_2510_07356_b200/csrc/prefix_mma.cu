@@ -172,11 +172,11 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                             mbar_arrive_expect_tx(full_k(s), npages * box_bytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
-                                if (q < npages) tma_load_tile(kdst + q * box_bytes, &map_k, (pages[q] * kHkv + g) * p.page_size + row_in_page, full_k(s));
+                                if (q < npages) tma_load_tile(kdst + q * box_bytes, &map_k, pool_row(p, pages[q], g, row_in_page), full_k(s), pool_plane(p, g));
                             mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
                             #pragma unroll
                             for (int q = 0; q < 4; ++q)
-                                if (q < npages) tma_load_tile(vdst + q * box_bytes, &map_v, (pages[q] * kHkv + g) * p.page_size + row_in_page, full_v(s));
+                                if (q < npages) tma_load_tile(vdst + q * box_bytes, &map_v, pool_row(p, pages[q], g, row_in_page), full_v(s), pool_plane(p, g));
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -433,11 +433,12 @@ EncodeTiledFn encode_fn() {
 
 // Rows of 128 bf16 seen as {64 elements, rows, 2 halves}; a box of `box_rows` rows lands in
 // shared memory as [half][row][128 B] with the 128-byte swizzle.
-bool make_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows) {
+bool make_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int planes = 2) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {64, rows, 2};
-    const cuuint64_t strides[2] = {256, 128};
+    // planes = 2: rows of 128 elements; planes = 16: token-major pool rows (8 heads x 2 halves per token)
+    const cuuint64_t dims[3] = {64, rows, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)planes * 128, 128};
     const cuuint32_t box[3] = {64, box_rows, 2};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -459,8 +460,10 @@ cudaError_t launch_ns(const DecodeParams& p, const CascadeParams& c, const CUten
 
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
-    const uint64_t pool_rows = (uint64_t)p.num_pages * kHkv * p.page_size;
-    if (!make_row_map(&mk, p.k_pages, pool_rows, p.box_rows) || !make_row_map(&mv, p.v_pages, pool_rows, p.box_rows) ||
+    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
+    const int planes = p.token_major ? 2 * kHkv : 2;
+    if (!make_row_map(&mk, p.k_pages, pool_rows, p.box_rows, planes) ||
+        !make_row_map(&mv, p.v_pages, pool_rows, p.box_rows, planes) ||
         !make_row_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup))
         return cudaErrorInvalidValue;
     return launch_ns<kMaxShare>(p, c, mk, mv, mq, stream);

@@ -56,11 +56,12 @@ __device__ __forceinline__ void wait_failed(const DecodeParams& p, volatile int3
     atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagWaitLimit);
     atomicCAS(p.hdr + kHdrWaitSite, 0, site);
 }
-__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int32_t row, uint32_t bar) {
-    // box {64 elements, P rows, 2 halves} at coordinates {0, row, 0}
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int32_t row, uint32_t bar,
+                                              int32_t plane = 0) {
+    // box {64 elements, P rows, 2 halves} at coordinates {0, row, plane}
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(bar) : "memory");
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(plane), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile(
