@@ -30,6 +30,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace concur {
 
@@ -65,7 +66,6 @@ struct CombineJob {
 
 struct Smem {
     // offsets from the 1024-aligned base
-    static constexpr int kStagesOff = 0;
     static constexpr int kMergeOff = kStages * kStageBytes;
     static constexpr int kMlOff = kMergeOff + kMergeBytes;                       // [4 warps][8 heads][2]
     static constexpr int kPrefixOff = kMlOff + kConsumerWarps * kGroup * 2 * 4;  // [kSmemBatch + 1]
@@ -543,44 +543,6 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
 
 // ------------------------------------------------------------------ host side
 
-namespace {
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            sym = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(sym);
-    }();
-    return fn;
-}
-
-// A pool [num_pages][8][P][128] bf16 seen as {64 elements, rows, 2 halves}: element stride 2 B,
-// row stride 256 B, half stride 128 B.  A box {64, P, 2} is one (page, head) chunk and lands in
-// shared memory as [half][row][128 B] with the 128-byte swizzle.
-bool make_pool_map(CUtensorMap* map, const void* pool, int32_t num_pages, int32_t P, int32_t token_major) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    // token-major pools [page][slot][8][128]: a row (token) is 2 KB apart and the 16 half-planes of
-    // its 8 heads are 128 B apart; the box is the same {64, rows, 2}, at plane 2 g
-    const cuuint64_t dims[3] = {64, token_major ? (cuuint64_t)num_pages * P : (cuuint64_t)num_pages * kHkv * P,
-                                token_major ? (cuuint64_t)(2 * kHkv) : 2};
-    const cuuint64_t strides[2] = {token_major ? (cuuint64_t)(kHkv * 256) : 256, 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)(P < kTile ? P : kTile), 2};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pool), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-}  // namespace
-
 cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
     static bool attr_set[64] = {};
     int dev = 0;
@@ -595,8 +557,11 @@ cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
         if (e != cudaSuccess) return e;
     }
     CUtensorMap map_k, map_v;
-    if (!make_pool_map(&map_k, p.k_pages, p.num_pages, p.page_size, p.token_major) ||
-        !make_pool_map(&map_v, p.v_pages, p.num_pages, p.page_size, p.token_major))
+    // one box {64, rows of a box, 2} = the part of one (page, KV head) chunk that belongs to a tile
+    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
+    const uint32_t planes = p.token_major ? 2 * kHkv : 2;
+    if (!make_rows_map(&map_k, p.k_pages, pool_rows, p.box_rows, 2, planes) ||
+        !make_rows_map(&map_v, p.v_pages, pool_rows, p.box_rows, 2, planes))
         return cudaErrorInvalidValue;
     // programmatic dependent launch: the prologue (barrier set-up) may overlap the plan kernel
     cudaLaunchConfig_t cfg = {};

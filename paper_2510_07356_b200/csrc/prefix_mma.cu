@@ -22,6 +22,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace concur {
 
@@ -415,37 +416,6 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
 
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            sym = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(sym);
-    }();
-    return fn;
-}
-
-// Rows of 128 bf16 seen as {64 elements, rows, 2 halves}; a box of `box_rows` rows lands in
-// shared memory as [half][row][128 B] with the 128-byte swizzle.
-bool make_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows, int planes = 2) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    // planes = 2: rows of 128 elements; planes = 16: token-major pool rows (8 heads x 2 halves per token)
-    const cuuint64_t dims[3] = {64, rows, (cuuint64_t)planes};
-    const cuuint64_t strides[2] = {(cuuint64_t)planes * 128, 128};
-    const cuuint32_t box[3] = {64, box_rows, 2};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int NS>
 cudaError_t launch_ns(const DecodeParams& p, const CascadeParams& c, const CUtensorMap& mk, const CUtensorMap& mv,
                       const CUtensorMap& mq, cudaStream_t stream) {
@@ -461,10 +431,10 @@ cudaError_t launch_ns(const DecodeParams& p, const CascadeParams& c, const CUten
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
     const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
-    const int planes = p.token_major ? 2 * kHkv : 2;
-    if (!make_row_map(&mk, p.k_pages, pool_rows, p.box_rows, planes) ||
-        !make_row_map(&mv, p.v_pages, pool_rows, p.box_rows, planes) ||
-        !make_row_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup))
+    const uint32_t planes = p.token_major ? 2 * kHkv : 2;
+    if (!make_rows_map(&mk, p.k_pages, pool_rows, p.box_rows, 2, planes) ||
+        !make_rows_map(&mv, p.v_pages, pool_rows, p.box_rows, 2, planes) ||
+        !make_rows_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup, 2))
         return cudaErrorInvalidValue;
     return launch_ns<kMaxShare>(p, c, mk, mv, mq, stream);
 }
