@@ -123,3 +123,17 @@ def test_cascade_argument_errors(P):
                                       check=False)
     assert rc == B.CONCUR_ERR_UNSUPPORTED
     big.close()
+
+
+@pytest.mark.parametrize("name,nseq", [("casc_24x10_pre2048_p64", 12), ("casc_16x10_pre16384_p64", 6)])
+def test_bench_workloads_on_sampled_sequences(P, name, nseq):
+    # the workloads bench.py times, in its launch configuration; the oracle on a seeded sample of sequences
+    cw = synth.make_named_cascade(name, "cuda:0")
+    out, lse, attn = run_cascade(P, cw)
+    assert attn.status() == 0
+    rng = np.random.default_rng(11)
+    seqs = sorted(rng.choice(cw.w.spec.batch, size=nseq, replace=False).tolist())
+    ref_out, ref_lse = oracle_sequences(synth.gather_sequences(cw.w, seqs))
+    idx = torch.as_tensor(seqs, device="cuda:0")
+    assert_parity(out[idx], lse[idx], ref_out, ref_lse, f"{name}, sampled sequences")
+    attn.close()

@@ -120,3 +120,12 @@ def test_argument_errors(P):
     assert call(tq=-1) == B.CONCUR_ERR_INVALID_ARG
     torch.cuda.synchronize()
     attn.close()
+
+
+@pytest.mark.parametrize("name", ["prefill_16x2048_p64", "prefill_chunk_8x2048_of_16384_p64"])
+def test_bench_workloads_on_sampled_tokens(P, name):
+    # the workloads bench.py times; the oracle on a seeded sample of query tokens
+    pw = synth.make_named_prefill(name, "cuda:0")
+    rng = np.random.default_rng(13)
+    tokens = sorted(set([0, pw.total_q - 1] + rng.integers(0, pw.total_q, 24).tolist()))
+    check(P, pw, tokens=tokens, what=name)
