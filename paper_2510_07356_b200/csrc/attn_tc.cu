@@ -411,8 +411,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                         const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
                         umma_ts(tmem_base + kTmemS + g * kTile, tmem_base + kTmemQ + k16 * 8, b, idesc_qk, k16 > 0);
                     }
-                    umma_commit(s_full(g));
-                    umma_commit(empty_k(ks));                               // that K stage may be overwritten
+                    umma_commit(s_full(g));       // (the K stage is released by the softmax group that sees this)
                     if (idx == cnt - 1) umma_commit(qt_free);              // the segment's last read of its queries
                 }
                 __syncwarp();
@@ -520,6 +519,10 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             if (mine) {
                 const bool first = mt.idx < 2;                   // this group's first tile of the segment
                 if (!mbar_wait(s_full(g), k & 1u, abort_flag)) { ok = false; site = 38; break; }
+                // Q.K^T of this tile is complete, so its K stage may be overwritten.  The release is a
+                // plain arrival from a thread that learns of the completion anyway: a second
+                // tcgen05.commit would cost the issuing thread about as much as an MMA.
+                if (row == 0) mbar_arrive(empty_k(it % kTKStages));
                 tc_fence_after_sync();
                 uint32_t pk[32];                                 // the row's 64 probabilities, bf16 pairs
                 float sum = 0.f, alpha = 1.f, m_use = m_ref;
