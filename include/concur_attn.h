@@ -82,6 +82,10 @@ typedef enum {
 #define CONCUR_OPT_PREFIX_KERNEL 10 /* shared-prefix pass of the cascade step: 0 (default) = tcgen05 kernel with
                                        TMEM accumulators, 1 = warp-level mma.sync kernel                 */
 
+#define CONCUR_OPT_SMALL_PAGE_COPY 11 /* tensor-core partial kernel with 16- or 32-token pages: 1 (default) = the
+                                        producer warp copies tiles 16 bytes per lane, 0 = one TMA box per
+                                        (page, head) chunk                                               */
+
 /* Layouts of the K and V pools (concur_attn_config_t.kv_layout). */
 #define CONCUR_KV_HEAD_MAJOR  0   /* [num_pages][Hkv][P][D]: one (page, head) tile is contiguous (default) */
 #define CONCUR_KV_TOKEN_MAJOR 1   /* [num_pages][P][Hkv][D]: one token's rows of all KV heads are contiguous */

@@ -35,6 +35,7 @@ CONCUR_OPT_EVENT_AFTER_PARTIAL = 7
 CONCUR_OPT_FUSE_COMBINE = 8
 CONCUR_OPT_CLAIM_AHEAD = 9
 CONCUR_OPT_PREFIX_KERNEL = 10
+CONCUR_OPT_SMALL_PAGE_COPY = 11
 
 EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",

@@ -87,6 +87,7 @@ struct concur_attn {
     int32_t fuse_combine = 1;
     int32_t claim_ahead = 1 << 20;
     int32_t prefix_kernel = 0;
+    int32_t small_page_copy = 1;
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;
     Staging st_q, st_k, st_v, st_bt, st_len, st_out, st_lse;
     Staging cascade_ws;          // allocated on the first cascade call
@@ -153,6 +154,7 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.page_shift = h->cfg.page_size == 16 ? 4 : (h->cfg.page_size == 32 ? 5 : (h->cfg.page_size == 64 ? 6 : 7));
     p.box_rows = h->cfg.page_size < kTile ? h->cfg.page_size : kTile;
     p.box_shift = p.page_shift < 6 ? p.page_shift : 6;
+    p.lane_copy = p.box_rows < kTile ? h->small_page_copy : 0;
     p.token_major = h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0;
     p.hq = h->cfg.num_q_heads;
     p.group = h->cfg.num_q_heads / kHkv;
@@ -441,6 +443,9 @@ int concur_attn_set_option(concur_attn_t* h, int32_t key, int64_t value) {
         case CONCUR_OPT_PREFIX_KERNEL:
             if (value > 1) return CONCUR_ERR_INVALID_ARG;
             h->prefix_kernel = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_SMALL_PAGE_COPY:
+            if (value > 1) return CONCUR_ERR_INVALID_ARG;
+            h->small_page_copy = (int32_t)value; return CONCUR_OK;
         case CONCUR_OPT_EVENT_BEFORE_PARTIAL:
             h->ev_before = reinterpret_cast<cudaEvent_t>(static_cast<uintptr_t>(value)); return CONCUR_OK;
         case CONCUR_OPT_EVENT_AFTER_PARTIAL:

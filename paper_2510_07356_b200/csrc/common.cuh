@@ -46,6 +46,8 @@ struct DecodeParams {
     int32_t page_shift;       // log2(page_size)
     int32_t box_rows;         // rows of one TMA box = min(page_size, 64): a 64-token tile is 64 / box_rows boxes
     int32_t box_shift;        // log2(box_rows)
+    int32_t lane_copy;        // tensor-core partial kernel, box_rows < 64: 1 = tiles are brought in by per-lane
+                              // 16-byte asynchronous copies instead of one TMA box per (page, head) chunk
     int32_t token_major;      // 0: pools are [page][KV head][slot][D]; 1: [page][slot][KV head][D]
     int32_t group;            // query heads per KV head (1..kGroup); heads g*group .. g*group+group-1 share KV head g
     int32_t hq;               // query heads = kHkv * group

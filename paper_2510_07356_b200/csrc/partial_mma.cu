@@ -40,7 +40,9 @@ constexpr int kStages = 6;
 constexpr int kConsumerWarps = 4;
 constexpr int kProducerWarp = kConsumerWarps;          // warp 4
 constexpr int kCombinerWarp = kConsumerWarps + 1;      // warp 5
-constexpr int kThreads = (kConsumerWarps + 2) * 32;
+constexpr int kCopyWarp0 = kConsumerWarps + 2;         // warps 6-8: copy helpers, used with small pages only
+constexpr int kCopyWarps = 3;
+constexpr int kThreads = (kConsumerWarps + 2 + kCopyWarps) * 32;
 constexpr int kTileBytes = kTile * kRowBytes;             // 16 KB: one K or V tile
 constexpr int kQBytes = kGroup * kRowBytes;               // 2 KB: the 8 query rows of a group
 constexpr int kStageBytes = 2 * kTileBytes + kQBytes;     // K | V | Q
@@ -54,6 +56,7 @@ struct StageMeta {
     int32_t first, last;   // first / last tile of its segment
     int32_t unit_start;    // flat tile index of the unit's first tile
     int32_t tiles_b;       // tiles of the whole unit
+    int32_t page[4];       // small pages: pool pages of the tile's boxes (for the copy helpers)
 };
 
 // A finished partial segment handed from the consumer warps to the combiner warp.
@@ -71,8 +74,8 @@ struct Smem {
     static constexpr int kPrefixOff = kMlOff + kConsumerWarps * kGroup * 2 * 4;  // [kSmemBatch + 1]
     static constexpr int kLenOff = kPrefixOff + (kSmemBatch + 1) * 4;            // [kSmemBatch + 1]
     static constexpr int kMetaOff = kLenOff + (kSmemBatch + 1) * 4;
-    static constexpr int kBarOff = kMetaOff + kStages * (int)sizeof(StageMeta);  // full_k, full_v, empty, merge x2, job x2
-    static constexpr int kAbortOff = kBarOff + (3 * kStages + 4) * 8;            // abort flag
+    static constexpr int kBarOff = kMetaOff + kStages * (int)sizeof(StageMeta);  // full_k, full_v, empty, merge x2, job x2, sched
+    static constexpr int kAbortOff = kBarOff + (4 * kStages + 4) * 8;            // abort flag
     static constexpr int kJobOff = kAbortOff + 16;                               // CombineJob
     static constexpr int kTotal = kJobOff + 32;
 };
@@ -101,6 +104,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     const uint32_t merge_bar1 = merge_bar0 + 8u;
     const uint32_t job_ready = merge_bar0 + 16u;      // consumers -> combiner: a job is posted
     const uint32_t job_taken = merge_bar0 + 24u;      // combiner -> consumers: the job slot is free again
+    auto sched = [&](int s) { return merge_bar0 + 32u + 8u * s; };   // producer -> copy helpers: the stage's record is written
     volatile CombineJob* job_s = reinterpret_cast<volatile CombineJob*>(smem + Smem::kJobOff);
 
     const int tid = threadIdx.x;
@@ -108,11 +112,19 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     const int32_t P = p.box_rows;            // rows per box: the unit of the shared-memory tile layout
     const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
     const bool cached = p.batch <= kSmemBatch;
+    // Small pages (16 or 32 tokens): a tile would be four or two TMA boxes per operand, and the copy
+    // engine's cost per box caps the stream well below HBM speed.  There the producer warp and three
+    // helper warps copy a quarter of the tile each (16 rows), 16 bytes per lane and instruction, into
+    // the same swizzled layout; a tile's barrier then takes one arrival per copying lane (when that
+    // lane's copies have landed) next to the producer's own.
+    const bool lane_copy = p.lane_copy != 0;
+    constexpr uint32_t kCopyLanes = (1 + kCopyWarps) * 32;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_k(s), 1);
-            mbar_init(full_v(s), 1);
+            mbar_init(full_k(s), lane_copy ? 1 + kCopyLanes : 1);
+            mbar_init(full_v(s), lane_copy ? kCopyLanes : 1);
+            mbar_init(sched(s), 1);
             mbar_init(empty(s), kConsumerWarps);
         }
         mbar_init(merge_bar0, kConsumerWarps * 32);
@@ -144,6 +156,50 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     }
     __syncthreads();
     const int32_t* prefix = cached ? sm_prefix : p.tiles_prefix;
+
+    // lane_copy: one instruction moves two 256-byte rows (lanes 0-15 the even row, 16-31 the odd
+    // one), 16-byte piece c16 of a row each.  In a box's [half][row][128 B] layout with the
+    // 128-byte swizzle, piece (half h, c) of row r sits at h*P*128 + r*128 + ((c ^ (r & 7)) << 4);
+    // for r = r0 + 2j + hi (r0 a multiple of 8) that is the per-lane term below + r0*128 + 256 j,
+    // with bits 4-6 xor-ed by (2j & 6).  Quarter w of a tile = its rows 16w .. 16w+15.
+    auto copy_quarter = [&](int s, int w, int32_t n_valid, int32_t g, int32_t page) {
+        const uint32_t hi = lane >> 4, c16 = lane & 15;
+        const uint32_t soff = (c16 >> 3) * (uint32_t)P * 128u + hi * 128u + (((c16 & 7u) ^ hi) << 4);
+        const uint32_t row_bytes = p.token_major ? (uint32_t)(kHkv * kRowBytes) : (uint32_t)kRowBytes;
+        const int32_t row0 = 16 * w;                              // first row of the quarter in its tile
+        const bool live = row0 < ((n_valid + P - 1) & ~(P - 1));  // whole boxes are read, as the TMA path does
+        const int32_t rb = row0 & (P - 1);                        // ... and in its page
+        const uint32_t d0 = smem_base + s * kStageBytes + (uint32_t)(row0 >> p.box_shift) * ((uint32_t)P * kRowBytes) +
+                            soff + (uint32_t)rb * 128u;
+        const int64_t e0 = pool_elem(p, page, g, rb) * 2 + hi * row_bytes + c16 * 16u;
+        #pragma unroll
+        for (int op = 0; op < 2; ++op) {                          // K, then V
+            if (live) {
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(op == 0 ? p.k_pages : p.v_pages) + e0;
+                const uint32_t d = d0 + op * kTileBytes;
+                #pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    lane_copy16((d + j * 256u) ^ ((2u * j & 6u) << 4), src + (size_t)(2 * j) * row_bytes);
+            }
+            lane_copy_arrive(op == 0 ? full_k(s) : full_v(s));
+        }
+    };
+
+    if (warp >= kCopyWarp0) {
+        // =========================================================== copy helper warps (small pages)
+        if (!lane_copy) return;
+        const int w = warp - kCopyWarp0 + 1;
+        for (uint32_t it = 0;; ++it) {
+            const int s = it % kStages;
+            if (!mbar_wait(sched(s), (it / kStages) & 1u, abort_flag)) {
+                if (lane == 0) wait_failed(p, abort_flag, 10);
+                return;
+            }
+            const int32_t n_valid = meta[s].n_valid;
+            if (n_valid == 0) return;
+            copy_quarter(s, w, n_valid, meta[s].g, meta[s].page[(16 * w) >> p.box_shift]);
+        }
+    }
 
     if (warp == kProducerWarp) {
         // =========================================================== producer warp
@@ -213,27 +269,35 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                             m.b = sg.b; m.g = sg.g; m.slot = sg.slot; m.n_valid = n_valid;
                             m.first = (t == sg.tile0); m.last = (t == sg.tile1 - 1);
                             m.unit_start = unit_start; m.tiles_b = sg.tiles_b;
+                            m.page[0] = page0; m.page[1] = page1; m.page[2] = page2; m.page[3] = page3;
                             const uint32_t kdst = smem_base + s * kStageBytes;
                             const uint32_t vdst = kdst + kTileBytes;
                             const bool with_q = (t == sg.tile0);
                             const uint32_t q_bytes = (uint32_t)p.group * kRowBytes;
-                            mbar_arrive_expect_tx(full_k(s), npages * box_bytes + (with_q ? q_bytes : 0));
+                            const uint32_t tile_tx = lane_copy ? 0u : npages * box_bytes;
+                            const uint32_t tx = tile_tx + (with_q ? q_bytes : 0);
+                            if (tx) mbar_arrive_expect_tx(full_k(s), tx);
+                            else mbar_arrive(full_k(s));
                             if (with_q)
                                 bulk_load(vdst + kTileBytes, p.q + ((int64_t)sg.b * p.hq + sg.g * p.group) * kD,
                                           q_bytes, full_k(s));
-                            const int32_t pages[4] = {page0, page1, page2, page3};
-                            #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                if (i < npages)
-                                    tma_load_tile(kdst + i * box_bytes, &map_k, pool_row(p, pages[i], sg.g, row_in_page), full_k(s), pool_plane(p, sg.g));
-                            mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
-                            #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                if (i < npages)
-                                    tma_load_tile(vdst + i * box_bytes, &map_v, pool_row(p, pages[i], sg.g, row_in_page), full_v(s), pool_plane(p, sg.g));
+                            if (lane_copy) mbar_arrive(sched(s));          // the helpers may read the record
+                            if (!lane_copy) {
+                                const int32_t pages[4] = {page0, page1, page2, page3};
+                                #pragma unroll
+                                for (int i = 0; i < 4; ++i)
+                                    if (i < npages)
+                                        tma_load_tile(kdst + i * box_bytes, &map_k, pool_row(p, pages[i], sg.g, row_in_page), full_k(s), pool_plane(p, sg.g));
+                                mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
+                                #pragma unroll
+                                for (int i = 0; i < 4; ++i)
+                                    if (i < npages)
+                                        tma_load_tile(vdst + i * box_bytes, &map_v, pool_row(p, pages[i], sg.g, row_in_page), full_v(s), pool_plane(p, sg.g));
+                            }
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (ok && lane_copy) copy_quarter(s, 0, n_valid, sg.g, page0);
                     if (ok) ++it;
                 }
             }
@@ -247,7 +311,8 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 ok = mbar_wait(empty(s), parity ^ 1u, abort_flag);
                 if (ok) {
                     meta[s].n_valid = 0;
-                    mbar_arrive(full_k(s));
+                    mbar_arrive_n(full_k(s), lane_copy ? 1 + kCopyLanes : 1);
+                    if (lane_copy) mbar_arrive(sched(s));
                 }
             }
             if (!ok) {

@@ -51,6 +51,33 @@ def test_plain_step(P, kernel, page_size, ranges, hq):
     attn.close()
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("page_size,ranges,hq", [(16, 0, 64), (16, 9, 40), (32, 0, 64), (32, 300, 24)])
+def test_small_pages_through_tma_boxes(P, layout, page_size, ranges, hq):
+    """With 16- and 32-token pages the tensor-core kernel's producer copies tiles lane by lane by
+    default; the alternative (one TMA box per page and head) must give the same results."""
+    spec = synth.tiny_spec(f"box_p{page_size}", LENS, page_size, 8200 + page_size, num_q_heads=hq)
+    w = synth.make_workload(spec, "cuda:0")
+    k, v = (token_major(w.k_pages), token_major(w.v_pages)) if layout else (w.k_pages, w.v_pages)
+    ref_out, ref_lse = oracle_sequences(host(w))
+    outs = []
+    for mode in (0, 1):
+        attn = P.DecodeAttention(page_size, spec.batch, w.block_table.shape[1], 0, num_q_heads=hq, kv_layout=layout)
+        attn.set_option(P.CONCUR_OPT_SMALL_PAGE_COPY, mode)
+        attn.set_option(P.CONCUR_OPT_NUM_RANGES, ranges)
+        out = torch.empty_like(w.q)
+        lse = torch.empty((spec.batch, hq), dtype=torch.float32, device="cuda:0")
+        P.concur_decode_attn(attn.handle, w.q, k, v, w.block_table, w.seq_lens, w.scale, out, lse, spec.batch,
+                             w.num_pages, w.block_table.shape[1], torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert attn.status() == 0
+        assert_parity(out, lse, ref_out, ref_lse, f"p{page_size} layout {layout} copy mode {mode}")
+        outs.append((out, lse))
+        attn.close()
+    # the two modes fill shared memory with the same bytes, so the arithmetic that follows is the same
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
 GROUPS = [(1024, [100, 1, 64, 700, 333]), (0, [500]), (2048, [5, 900]),
           (512, [0, 130, 64, 1, 2000, 77, 640, 63, 65, 300])]
 
