@@ -108,6 +108,24 @@ __device__ __forceinline__ int64_t pool_elem(const DecodeParams& p, int32_t page
                          : (((int64_t)page * kHkv + g) * p.page_size + slot) * kD;
 }
 
+// Number of split-KV ranges for W flat tiles: as many as keeps every CTA supplied `ranges_per_cta`
+// times over, but none shorter than `min_range_tiles`; or the forced count.  One definition, because
+// the plan kernel and a partial kernel that plans for itself must arrive at the same number.
+__device__ __forceinline__ int32_t plan_num_ranges(const DecodeParams& p, int32_t W) {
+    int32_t R;
+    if (p.forced_ranges > 0) {
+        R = p.forced_ranges;
+    } else {
+        R = W / p.min_range_tiles;
+        const int32_t cap = p.grid_ctas * p.ranges_per_cta;
+        if (R > cap) R = cap;
+    }
+    if (R > p.max_ranges) R = p.max_ranges;
+    if (R > W) R = W;
+    if (R < 1 && W > 0) R = 1;
+    return R;
+}
+
 // First flat tile of range r when [0, W) is cut into R ranges of equal size.
 __device__ __forceinline__ int32_t range_begin(int32_t W, int32_t R, int32_t r) {
     return (int32_t)(((int64_t)W * r) / R);

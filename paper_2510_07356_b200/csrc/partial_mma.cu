@@ -77,7 +77,8 @@ struct Smem {
     static constexpr int kBarOff = kMetaOff + kStages * (int)sizeof(StageMeta);  // full_k, full_v, empty, merge x2, job x2, sched
     static constexpr int kAbortOff = kBarOff + (4 * kStages + 4) * 8;            // abort flag
     static constexpr int kJobOff = kAbortOff + 16;                               // CombineJob
-    static constexpr int kTotal = kJobOff + 32;
+    static constexpr int kScanOff = kJobOff + 32;                                // per-warp totals of the tile scan
+    static constexpr int kTotal = kScanOff + 64;
 };
 constexpr int kSmemBytes = Smem::kTotal + 1024;           // slack for the manual 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
@@ -142,19 +143,68 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 make_uint4(0, 0, 0, 0);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    // everything above overlaps the plan kernel when launched as its programmatic dependent;
-    // the plan's outputs are read only below this wait
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int32_t W = p.hdr[kHdrTotalTiles];
-    const int32_t R = p.hdr[kHdrNumRanges];
-    if (cached) {
-        for (int i = tid; i <= p.batch; i += kThreads) sm_prefix[i] = p.tiles_prefix[i];
-        for (int i = tid; i < p.batch; i += kThreads) {
-            int64_t n = p.seq_lens[i];
-            sm_len[i] = (int32_t)(n < 0 ? 0 : (n > max_len ? max_len : n));
+    // Launched as the plan kernel's programmatic dependent, this kernel may run before the plan has
+    // finished.  In the plain step with a batch that fits the shared-memory tables it does not wait for
+    // it: the tile counts, their prefix and the range count follow from seq_lens alone, so every CTA
+    // works them out for itself (same arithmetic as the plan kernel) and starts streaming at once.
+    // What does depend on the plan kernel is its resets -- the claim counter and the per-unit ticket
+    // counters -- so each thread executes griddepcontrol.wait before its first atomic on either and
+    // before its first global store.  In the other modes the wait comes first and the tables are read.
+    const bool self_plan = cached && p.tok_offset == nullptr && !p.all_partial;
+    bool plan_seen = !self_plan;
+    int32_t W, R;
+    if (self_plan) {
+        int32_t* scan_ws = reinterpret_cast<int32_t*>(smem + Smem::kScanOff);
+        if (tid == 0) sm_prefix[0] = 0;
+        int32_t carry = 0;
+        for (int base = 0; base < p.batch; base += kThreads) {
+            const int b = base + tid;
+            int32_t v = 0;
+            if (b < p.batch) {
+                const int64_t nn = p.seq_lens[b];
+                const int32_t n = (int32_t)(nn < 0 ? 0 : (nn > max_len ? max_len : nn));
+                sm_len[b] = n;
+                v = (n + kTile - 1) / kTile;
+            }
+            #pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t up = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v += up;
+            }
+            if (lane == 31) scan_ws[warp] = v;
+            __syncthreads();
+            int32_t before = 0, total = 0;
+            #pragma unroll
+            for (int w2 = 0; w2 < kThreads / 32; ++w2) {
+                const int32_t x = scan_ws[w2];
+                total += x;
+                if (w2 < warp) before += x;
+            }
+            if (b < p.batch) sm_prefix[b + 1] = carry + before + v;
+            carry += total;
+            __syncthreads();
         }
+        W = kHkv * carry;
+        R = plan_num_ranges(p, W);
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        W = p.hdr[kHdrTotalTiles];
+        R = p.hdr[kHdrNumRanges];
+        if (cached) {
+            for (int i = tid; i <= p.batch; i += kThreads) sm_prefix[i] = p.tiles_prefix[i];
+            for (int i = tid; i < p.batch; i += kThreads) {
+                int64_t n = p.seq_lens[i];
+                sm_len[i] = (int32_t)(n < 0 ? 0 : (n > max_len ? max_len : n));
+            }
+        }
+        __syncthreads();
     }
-    __syncthreads();
+    auto see_plan = [&]() {
+        if (!plan_seen) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            plan_seen = true;
+        }
+    };
     const int32_t* prefix = cached ? sm_prefix : p.tiles_prefix;
 
     // lane_copy: one instruction moves two 256-byte rows (lanes 0-15 the even row, 16-31 the odd
@@ -235,7 +285,10 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 int32_t pg_next = (chunk_base + 32 + lane < page_end) ? __ldg(table + chunk_base + 32 + lane) : 0;
                 const int32_t unit_start = x - sg.tile1;      // x already points past the segment
                 for (int32_t t = sg.tile0; ok && t < sg.tile1; ++t) {
-                    if (!claimed && x1 - (unit_start + t) <= p.claim_ahead) {
+                    // (a CTA that has not waited for the plan kernel yet first fills its ring)
+                    if (!claimed && x1 - (unit_start + t) <= p.claim_ahead &&
+                        (plan_seen || unit_start + t - x0 >= kStages || unit_start + t == x1 - 1)) {
+                        see_plan();
                         if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
                         claimed = true;
                     }
@@ -337,6 +390,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         //   L = log2 sum_s 2^{lse_s},  out = sum_s 2^{lse_s - L} out_s,  lse = L ln 2
         // with a running maximum, 4 dims per lane, all 8 heads in flight at once.
         const float ninf_c = -INFINITY;
+        see_plan();
         for (uint32_t jobn = 0;; ++jobn) {
             if (!mbar_wait(job_ready, jobn & 1u, abort_flag)) {
                 if (lane == 0) wait_failed(p, abort_flag, 8);
@@ -536,6 +590,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
 
         if (mt.last) {
             // ---- merge the four warps' states and write the segment's result
+            see_plan();
             #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {
                 l0 += __shfl_xor_sync(0xffffffffu, l0, off);

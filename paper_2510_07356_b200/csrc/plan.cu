@@ -75,19 +75,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
 
     if (tid == 0) {
         const int32_t W = kHkv * carry_s;
-        int32_t R;
-        if (p.forced_ranges > 0) {
-            R = p.forced_ranges;
-        } else {
-            // as many ranges as keeps every CTA supplied `ranges_per_cta` times over,
-            // but none shorter than `min_range_tiles`
-            R = W / p.min_range_tiles;
-            int32_t cap = p.grid_ctas * p.ranges_per_cta;
-            if (R > cap) R = cap;
-        }
-        if (R > p.max_ranges) R = p.max_ranges;
-        if (R > W) R = W;
-        if (R < 1 && W > 0) R = 1;
+        const int32_t R = plan_num_ranges(p, W);
         p.hdr[kHdrTotalTiles] = W;
         p.hdr[kHdrNumRanges] = R;
         p.hdr[kHdrClaim] = p.grid_ctas;       // CTA i starts on range i; further ranges are claimed from here

@@ -106,6 +106,7 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.page_shift = page_size == 16 ? 4 : (page_size == 32 ? 5 : 6);
     p.box_rows = page_size;
     p.box_shift = p.page_shift;
+    p.lane_copy = page_size < kTile ? 1 : 0;
     p.hq = kHq;
     p.group = kGroup;
     p.grid_ctas = s->sm_count;

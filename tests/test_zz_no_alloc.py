@@ -26,16 +26,17 @@ def test_static_entry_matches_handle_entry_twice_in_a_row():
     # two different batches, the second one larger, so that anything the first call left in
     # the shared array would be noticed
     specs = [synth.tiny_spec("na0", (3000, 1, 0, 64, 777, 12000), 64, 501),
-             synth.tiny_spec("na1", (9000, 20000, 130, 64, 5, 0, 4100, 2500), 64, 502)]
+             synth.tiny_spec("na1", (9000, 20000, 130, 64, 5, 0, 4100, 2500), 64, 502),
+             synth.tiny_spec("na2", (700, 17, 0, 3000, 33), 16, 503)]
     for spec in specs:
         w = synth.make_workload(spec, "cuda:0")
         B = spec.batch
-        ref = P.DecodeAttention(64, B, w.block_table.shape[1], 0)
+        ref = P.DecodeAttention(spec.page_size, B, w.block_table.shape[1], 0)
         out_ref, lse_ref = ref(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
         out = torch.full_like(w.q, 7.0)
         lse = torch.full((B, 64), 7.0, dtype=torch.float32, device="cuda:0")
         P.concur_decode_attn_static(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale,
-                                    out, lse, B, w.num_pages, w.block_table.shape[1], 64, stream)
+                                    out, lse, B, w.num_pages, w.block_table.shape[1], spec.page_size, stream)
         torch.cuda.synchronize()
         a, b = out.float(), out_ref.float()
         assert torch.isfinite(a).all()
