@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one partial_mma_kernel launch divided by its KV tokens, from
 # the ncu capture summarised in profiles/partial_mma_cfg3q_b16_ctx16384.md (page size 64, fused combine, one
 # range per CTA).  Set to None whenever that kernel changes until the counters are taken again.
-MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074881e9 + 5.180672e6) / 262144
+MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074874e9 + 4.741888e6) / 262144
 
 
 def parse_args():
