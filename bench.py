@@ -39,6 +39,12 @@ FALLBACK_HBM_GBS = 6650.0
 # the ncu capture summarised in profiles/partial_mma_cfg3q_b16_ctx16384.md (page size 64, fused combine, one
 # range per CTA).  Set to None whenever that kernel changes until the counters are taken again.
 MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074874e9 + 4.741888e6) / 262144
+# The same two counters of one attn_tc_kernel launch on exactly these workloads (profiles/attn_tc_*.md); None for
+# any other workload, and to be removed whenever that kernel changes until the counters are taken again.
+ATTN_TC_TRAFFIC_BYTES = {
+    ("casc_16x10_pre16384_p64", "tcgen05"): 1.080155e9 + 11.060992e6,
+    ("prefill_16x2048_p64", "tcgen05"): 671.256320e6 + 506.075904e6,
+}
 
 
 def parse_args():
@@ -384,7 +390,9 @@ def run_cascade(args):
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "prefix pass", "ms": pre_ms_avg,
+                     "peak_kind": f"of {peak_kind}",
+                     "traffic": ATTN_TC_TRAFFIC_BYTES.get((args.workload, "tcgen05" if args.prefix_kernel == 0 else "mma.sync")),
+                     "kernel": "prefix pass", "ms": pre_ms_avg,
                      "ms_min": min(pre_ms)},
         "e2e": None, "gpu_launches": 4 * K, "clocks": clocks, "device_flags": flags,
     }
@@ -489,7 +497,8 @@ def run_prefill(args):
                    "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
         "query_tokens_per_s": job_q / (ms_per_step * 1e-3),
         "roofline": {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s",
-                     "frac": value / world / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "frac": value / world / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": ATTN_TC_TRAFFIC_BYTES.get((spec.name, "tcgen05")),
                      "kernel": "plan + attn_tc_kernel<prefill>", "ms": ms_per_step, "ms_min": min(step_ms)},
         "e2e": None, "gpu_launches": 2 * K, "clocks": clocks, "device_flags": flags,
     }
