@@ -241,7 +241,8 @@ def cpu_baseline(w, target_seconds, results=None):
     nbytes = sub.algorithmic_bytes()
     base = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{len(seqs)} of {w.spec.batch} sequences ({tok} of {w.kv_tokens} KV tokens), all {w.spec.num_q_heads} query heads, "
-                      f"{dt:.1f} s wall", "kv_tokens_per_s": tok / dt}
+                      f"{dt:.1f} s wall", "kv_tokens_per_s": tok / dt,
+            "one_core_kv_tokens_per_s": 1.0 / max(per_token_core, 1e-12)}      # from the calibration call
     if results is None:
         return base
     return base, parity_of(rows, seqs, results[0], results[1])
@@ -852,7 +853,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": spec.name, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
+        "config": {"workload": spec.name, "seed": spec.seed, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
                    "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128, "algorithmic_bytes": nbytes,
                    "l2": "flushed between steps (256 MB written, then 256 MB read)" if flush_needed else "inputs larger than L2",
                    "kernel": "mma" if args.kernel == 0 else "scalar", "ranges": R, "tiles": W,

@@ -265,6 +265,27 @@ def test_many_short_sequences(P, kernel):
     attn.close()
 
 
+@pytest.mark.parametrize("batch", [288, 289, 300, 511, 512])
+@pytest.mark.parametrize("page_size,ranges", [(64, 0), (16, 37)])
+def test_batch_sizes_around_the_in_kernel_plan_limits(P, batch, page_size, ranges):
+    # up to 511 sequences the tensor-core kernel derives the tile prefix and the range count from
+    # seq_lens itself (288 threads per scan round: one round, two rounds, the last cached batch);
+    # from 512 on it reads the plan kernel's tables.  Both must cut the same ranges.
+    rng = np.random.default_rng(4000 + batch)
+    lens = rng.integers(0, 300, size=batch)
+    lens[rng.integers(0, batch, size=20)] = 0
+    lens[batch - 1] = 777                                  # the last sequence matters to the scan's tail
+    spec = synth.tiny_spec(f"plan{batch}", [int(x) for x in lens], page_size, 4100 + batch)
+    w = synth.make_workload(spec, "cuda:0")
+    out, lse, attn = run(P, w, 0, ranges)
+    assert attn.status() == 0
+    R, W, starts = attn.last_plan()
+    assert W == 8 * sum(-(-int(n) // 64) for n in lens)
+    ref_out, ref_lse = oracle_sequences(to_host(w))
+    assert_parity(out, lse, ref_out, ref_lse, f"batch {batch} p{page_size} R{ranges}")
+    attn.close()
+
+
 def test_repeated_calls_on_one_handle_are_identical(P):
     # the workspace is reused call after call: counters and partial slots of an earlier,
     # larger call must not leak into a later one
