@@ -67,7 +67,9 @@ typedef enum {
 #define CONCUR_OPT_KERNEL      1    /* 0 = tensor-core partial kernel (default), 1 = scalar-FMA kernel */
 #define CONCUR_OPT_NUM_RANGES  2    /* force the number of split-KV ranges; 0 = heuristic              */
 #define CONCUR_OPT_GRID_CTAS   3    /* force the partial kernel's grid size; 0 = one wave of the GPU    */
-#define CONCUR_OPT_RANGES_PER_CTA 4 /* heuristic's target ranges per CTA; 0 = built-in default (1)      */
+#define CONCUR_OPT_RANGES_PER_CTA 4 /* heuristic's target ranges per CTA; 0 = built-in default: 1, or 2 for a
+                                       skewed batch (longest sequence >= 4 x the mean) whose ranges then
+                                       still have 64 tiles or more                                       */
 #define CONCUR_OPT_MIN_RANGE_TILES 5/* heuristic's smallest range, in 64-token tiles; 0 = default (2)   */
 #define CONCUR_OPT_EVENT_BEFORE_PARTIAL 6 /* a cudaEvent_t (as an integer) recorded on the call's stream
                                              just before the partial kernel; 0 = none.  For timing

@@ -161,7 +161,7 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     const int per_sm = h->kernel == 1 ? partial_scalar_ctas_per_sm() : 1;
     p.grid_ctas = h->grid_ctas > 0 ? h->grid_ctas : h->sm_count * per_sm;
     p.forced_ranges = h->forced_ranges;
-    p.ranges_per_cta = h->ranges_per_cta > 0 ? h->ranges_per_cta : 1;
+    p.ranges_per_cta = h->ranges_per_cta;                 // 0: chosen per call from the amount of work
     p.min_range_tiles = h->min_range_tiles > 0 ? h->min_range_tiles : 2;
     p.max_ranges = kMaxRanges;
     p.fuse_combine = h->fuse_combine;

@@ -111,13 +111,23 @@ __device__ __forceinline__ int64_t pool_elem(const DecodeParams& p, int32_t page
 // Number of split-KV ranges for W flat tiles: as many as keeps every CTA supplied `ranges_per_cta`
 // times over, but none shorter than `min_range_tiles`; or the forced count.  One definition, because
 // the plan kernel and a partial kernel that plans for itself must arrive at the same number.
-__device__ __forceinline__ int32_t plan_num_ranges(const DecodeParams& p, int32_t W) {
+// `max_tiles` is the tile count of the longest sequence.
+__device__ __forceinline__ int32_t plan_num_ranges(const DecodeParams& p, int32_t W, int32_t max_tiles) {
     int32_t R;
     if (p.forced_ranges > 0) {
         R = p.forced_ranges;
     } else {
         R = W / p.min_range_tiles;
-        const int32_t cap = p.grid_ctas * p.ranges_per_cta;
+        // Ranges per CTA: the caller's, or (0) one -- but two for a skewed batch (the longest sequence
+        // four times the mean or more) with 64 tiles or more left per range.  Ranges hold equal
+        // numbers of tiles, but every (sequence, KV head) unit that ends inside one also costs a merge
+        // worth about three tiles; when unit lengths differ much, so do these sums, and a CTA that
+        // finishes early then takes a second range off one that does not.  On even batches the
+        // second range only costs its start-up.
+        const bool skewed = (int64_t)max_tiles * kHkv * p.batch >= 4 * (int64_t)W;
+        const int32_t per_cta = p.ranges_per_cta > 0 ? p.ranges_per_cta
+                                                     : (skewed && W >= p.grid_ctas * 2 * 64 ? 2 : 1);
+        const int32_t cap = p.grid_ctas * per_cta;
         if (R > cap) R = cap;
     }
     if (R > p.max_ranges) R = p.max_ranges;

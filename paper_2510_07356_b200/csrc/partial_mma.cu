@@ -78,7 +78,7 @@ struct Smem {
     static constexpr int kAbortOff = kBarOff + (4 * kStages + 4) * 8;            // abort flag
     static constexpr int kJobOff = kAbortOff + 16;                               // CombineJob
     static constexpr int kScanOff = kJobOff + 32;                                // per-warp totals of the tile scan
-    static constexpr int kTotal = kScanOff + 64;
+    static constexpr int kTotal = kScanOff + 128;
 };
 constexpr int kSmemBytes = Smem::kTotal + 1024;           // slack for the manual 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
@@ -156,7 +156,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     if (self_plan) {
         int32_t* scan_ws = reinterpret_cast<int32_t*>(smem + Smem::kScanOff);
         if (tid == 0) sm_prefix[0] = 0;
-        int32_t carry = 0;
+        int32_t carry = 0, longest = 0;
         for (int base = 0; base < p.batch; base += kThreads) {
             const int b = base + tid;
             int32_t v = 0;
@@ -166,12 +166,15 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 sm_len[b] = n;
                 v = (n + kTile - 1) / kTile;
             }
+            int32_t mx = v;
+            #pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int32_t up = __shfl_up_sync(0xffffffffu, v, o);
                 if (lane >= o) v += up;
             }
-            if (lane == 31) scan_ws[warp] = v;
+            if (lane == 31) { scan_ws[warp] = v; scan_ws[kThreads / 32 + warp] = mx; }
             __syncthreads();
             int32_t before = 0, total = 0;
             #pragma unroll
@@ -179,13 +182,14 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 const int32_t x = scan_ws[w2];
                 total += x;
                 if (w2 < warp) before += x;
+                longest = max(longest, scan_ws[kThreads / 32 + w2]);
             }
             if (b < p.batch) sm_prefix[b + 1] = carry + before + v;
             carry += total;
             __syncthreads();
         }
         W = kHkv * carry;
-        R = plan_num_ranges(p, W);
+        R = plan_num_ranges(p, W, longest);
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");
         W = p.hdr[kHdrTotalTiles];

@@ -15,13 +15,14 @@ constexpr int kPlanThreads = 1024;
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
     __shared__ int32_t warp_sums[kPlanThreads / 32];
     __shared__ int32_t carry_s;
+    __shared__ int32_t max_s;
     __shared__ int32_t ranges_s;
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     // lets a dependent launch (programmatic stream serialisation) start its prologue now; it
     // still waits for this grid to finish before it reads the plan
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid == 0) { carry_s = 0; p.tiles_prefix[0] = 0; }
+    if (tid == 0) { carry_s = 0; max_s = 0; p.tiles_prefix[0] = 0; }
     __syncthreads();
 
     const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
@@ -45,6 +46,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
             for (int i = lane; i < p.hq * kD / 8; i += 32) o[i] = make_uint4(0, 0, 0, 0);
             for (int i = lane; i < p.hq; i += 32) p.lse[(int64_t)e * p.hq + i] = -INFINITY;
         }
+        // the longest sequence (for the range-count heuristic)
+        int32_t mx = tiles;
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0 && mx > 0) atomicMax(&max_s, mx);
         // inclusive scan over the block
         int32_t v = tiles;
         #pragma unroll
@@ -75,7 +81,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
 
     if (tid == 0) {
         const int32_t W = kHkv * carry_s;
-        const int32_t R = plan_num_ranges(p, W);
+        const int32_t R = plan_num_ranges(p, W, max_s);
         p.hdr[kHdrTotalTiles] = W;
         p.hdr[kHdrNumRanges] = R;
         p.hdr[kHdrClaim] = p.grid_ctas;       // CTA i starts on range i; further ranges are claimed from here

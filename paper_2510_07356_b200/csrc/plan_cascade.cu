@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_cascade_kernel(DecodeParams
     __syncthreads();
     if (tid == 0) {
         const int32_t W = kHkv * carry;
-        int32_t R = p.forced_ranges > 0 ? p.forced_ranges : min(W / p.min_range_tiles, p.grid_ctas * p.ranges_per_cta);
+        int32_t R = p.forced_ranges > 0 ? p.forced_ranges : min(W / p.min_range_tiles, p.grid_ctas * (p.ranges_per_cta > 0 ? p.ranges_per_cta : 1));
         if (R > p.max_ranges) R = p.max_ranges;
         if (R > W) R = W;
         if (R < 1 && W > 0) R = 1;

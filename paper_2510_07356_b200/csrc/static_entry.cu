@@ -111,7 +111,7 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.group = kGroup;
     p.grid_ctas = s->sm_count;
     p.forced_ranges = 0;
-    p.ranges_per_cta = 1;
+    p.ranges_per_cta = 0;
     p.min_range_tiles = 2;
     p.max_ranges = kStaticMaxRanges;
     p.fuse_combine = 1;
