@@ -16,16 +16,18 @@
 //   O[128 x 128] += P[128 x 64] . V_tile[64 x 128]     (4 MMAs of K = 16; O in TMEM, V is the
 //                 MN-major B operand exactly as TMA laid it down)
 //
-// Both A operands live in TMEM: the queries are copied there once per segment (they do not
-// change from tile to tile) and P never leaves it, so the only shared-memory traffic of the
-// tensor pipe is one pass over the K tile and one over the V tile.  (With Q and P as
-// shared-memory operands the pipe spent ~1,100 clocks per tile fetching them -- more than the
-// HBM time of the tile.)
+// P never leaves TMEM (it is the A operand of P.V in the TS form).  The queries are the A operand of
+// Q.K^T in the SS form, read straight from the staging buffer the TMA copies fill -- 8-row groups of
+// 128-byte swizzled rows, which is the K-major operand layout as it stands.  (An earlier version
+// copied them into TMEM once per segment; that saved 32 KB of operand reads per tile, which the
+// tensor pipe does not miss, but tied the first product of a segment to the moment softmax group
+// A had finished the previous segment.  With P in shared memory as well, the pipe spent ~1,100
+// clocks per tile fetching operands.)
 //
 // One softmax warp per SM sub-partition is a serial chain (TMEM load, maximum, 64 exponentials
 // at 4 per clock, pack, store, fences) of about 1,900 clocks per tile, which is below the HBM
 // rate.  So there are TWO softmax warpgroups that take alternate tiles, each with its own
-// score buffer, P columns and O accumulator (TMEM columns: Q, S_A, S_B, P_A, P_B, O_A, O_B); while one group
+// score buffer, P columns and O accumulator (TMEM columns: S_A, S_B, P_A, P_B, O_A, O_B); while one group
 // is in its exponentials the other loads its scores.  At the end of a segment the two
 // (m, l, O) states of every row are merged by their log-sum-exp, each group writing half of
 // the output columns.
@@ -63,6 +65,8 @@ namespace {
 // Two uses of the same pipeline.  Prefix pass of the cascade step: a row group is a sibling (up to
 // kMaxShare = 10), every tile is whole and fully visible.  Prefill: a row group is a query token
 // (16 per unit), the tiles on the diagonal are masked causally and the last one may be ragged.
+constexpr int kTRows = 128;                               // MMA M
+
 template <bool kPrefill>
 struct TCfg {
     static constexpr int kShare = kPrefill ? 16 : kMaxShare;          // row groups (of 8 heads) per unit
@@ -71,6 +75,10 @@ struct TCfg {
     static constexpr int kQRows = kShare * kGroup;                    // query rows that are really loaded
     static constexpr int kQHalfBytes = kQRows * 128;
     static constexpr int kQBytes = 2 * kQHalfBytes;                   // per staging buffer
+    // Q.K^T reads its A operand straight from a staging buffer, always 128 rows of each half; where
+    // fewer rows are staged the read runs on into what follows the half.  Behind the last half that
+    // must still be this kernel's own, defined shared memory: a zeroed pad.
+    static constexpr int kQPad = kTRows * 128 > kQHalfBytes ? kTRows * 128 - kQHalfBytes : 0;
 };
 constexpr int kTVLag = 2;                                 // V of tile t is requested with K of tile t + 2
 constexpr int kTMetaRing = 16;                            // tile records; readers trail the producer by < 8
@@ -78,13 +86,12 @@ constexpr int kTProducerWarp = 8;
 constexpr int kTMmaWarp = 9;                              // issues Q.K^T, owns the TMEM allocation
 constexpr int kTPvWarp = 10;                              // issues P.V
 constexpr int kTThreads = 11 * 32;
-constexpr int kTRows = 128;                               // MMA M
 constexpr int kTHalfBytes = kTile * 128;                  // 8 KB: 64 tokens x one 64-dim half
 constexpr int kTTileBytes = 2 * kTHalfBytes;              // 16 KB: one K or V tile
-// TMEM columns (512): Q as packed bf16 [0,64); S_A [64,128), S_B [128,192); P_A [192,224),
-// P_B [224,256) as packed bf16; O_A [256,384), O_B [384,512)
+// TMEM columns (512): [0,64) free; S_A [64,128), S_B [128,192); P_A [192,224), P_B [224,256) as
+// packed bf16; O_A [256,384), O_B [384,512)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemQ = 0, kTmemS = 64, kTmemP = 192, kTmemO = 256;
+constexpr uint32_t kTmemS = 64, kTmemP = 192, kTmemO = 256;
 
 
 struct TMeta {
@@ -108,12 +115,12 @@ struct TSmem {
     static constexpr int kTKStages = Cfg::kKStages, kTVStages = Cfg::kVStages;
     static constexpr int kVOff = kTKStages * kTTileBytes;
     static constexpr int kQOff = kVOff + kTVStages * kTTileBytes;         // two staging buffers of the queries
-    static constexpr int kXchOff = kQOff + 2 * Cfg::kQBytes;              // [2 groups][128 rows] (m, l)
+    static constexpr int kXchOff = kQOff + 2 * Cfg::kQBytes + Cfg::kQPad; // [2 groups][128 rows] (m, l)
     static constexpr int kMetaOff = kXchOff + 2 * kTRows * 8;
     static constexpr int kBarOff = kMetaOff + kTMetaRing * (int)sizeof(TMeta);
     // full_k, empty_k per K stage; full_v, empty_v per V stage; meta_full per record; then pairs:
-    // q_full, q_empty, s_full, s_free, p_full, pv_done; xch_a, xch_b; qt_ready, qt_free
-    static constexpr int kNumBars = 2 * kTKStages + 2 * kTVStages + kTMetaRing + 16;
+    // q_full, q_empty, s_full, s_free, p_full, pv_done; xch_a, xch_b
+    static constexpr int kNumBars = 2 * kTKStages + 2 * kTVStages + kTMetaRing + 14;
     static constexpr int kTmemPtrOff = kBarOff + kNumBars * 8;
     static constexpr int kAbortOff = kTmemPtrOff + 8;
     static constexpr int kTotal = kAbortOff + 8;
@@ -140,7 +147,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
     using SM = TSmem<kPrefill>;
     using Cfg = TCfg<kPrefill>;
     constexpr int kTKStages = Cfg::kKStages, kTVStages = Cfg::kVStages;
-    constexpr int kTQRows = Cfg::kQRows, kTQHalfBytes = Cfg::kQHalfBytes, kTQBytes = Cfg::kQBytes;
+    constexpr int kTQHalfBytes = Cfg::kQHalfBytes, kTQBytes = Cfg::kQBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -163,15 +170,13 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
     auto pv_done = [&](int i) { return bar_base + 8u * (kB0 + 10 + i); };
     const uint32_t xch_a = bar_base + 8u * (kB0 + 12);               // both groups have published (m, l)
     const uint32_t xch_b = xch_a + 8u;                               // both groups have read both O
-    const uint32_t qt_ready = xch_a + 16u;                           // the segment's queries are in TMEM
-    const uint32_t qt_free = xch_a + 24u;                            // the segment's last Q.K^T has completed
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int32_t P = p.box_rows;            // rows per box: the unit of the shared-memory tile layout
 
     // unused query rows must at least be defined once
-    for (int i = tid; i < (2 * kTQBytes) / 16; i += kTThreads)
+    for (int i = tid; i < (2 * kTQBytes + Cfg::kQPad) / 16; i += kTThreads)
         reinterpret_cast<uint4*>(smem + SM::kQOff)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
         for (int s = 0; s < kTKStages; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
@@ -179,7 +184,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         for (int s = 0; s < kTMetaRing; ++s) mbar_init(meta_full(s), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(q_full(i), 1);
-            mbar_init(q_empty(i), 128);
+            mbar_init(q_empty(i), 1);                            // one commit after the segment's last Q.K^T
             mbar_init(s_full(i), 1);
             mbar_init(s_free(i), 128);
             mbar_init(p_full(i), 128);
@@ -187,8 +192,6 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         }
         mbar_init(xch_a, 256);
         mbar_init(xch_b, 256);
-        mbar_init(qt_ready, 128);
-        mbar_init(qt_free, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -396,23 +399,25 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                 const TMeta* mt = &meta[it % kTMetaRing];
                 const int32_t idx = mt->idx, cnt = mt->cnt;
                 if (mt->n == 0) break;
-                if (idx == 0) {                               // a segment starts: its queries must be in TMEM
-                    if (!mbar_wait(qt_ready, segs & 1u, abort_flag)) { ok = false; site = 33; break; }
+                if (idx == 0) {                               // a segment starts: its queries must have landed
+                    if (!mbar_wait(q_full(mt->qsel), (segs >> 1) & 1u, abort_flag)) { ok = false; site = 33; break; }
                     ++segs;
                 }
                 // the group has copied the scores of its previous tile out of the buffer
                 if (!mbar_wait(s_free(g), ((it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; site = 34; break; }
                 tc_fence_after_sync();
                 const uint32_t k_addr = smem_base + ks * kTTileBytes;
+                const uint32_t q_addr = smem_base + SM::kQOff + mt->qsel * kTQBytes;
                 if (lane == 0) {
                     #pragma unroll
                     for (int k16 = 0; k16 < 8; ++k16) {
                         const uint32_t koff = (uint32_t)(k16 & 3) * 32u;
+                        const uint64_t a = umma_smem_desc(q_addr + (k16 >> 2) * kTQHalfBytes + koff, 16, 1024);
                         const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
-                        umma_ts(tmem_base + kTmemS + g * kTile, tmem_base + kTmemQ + k16 * 8, b, idesc_qk, k16 > 0);
+                        umma_ss(tmem_base + kTmemS + g * kTile, a, b, idesc_qk, k16 > 0);
                     }
                     umma_commit(s_full(g));       // (the K stage is released by the softmax group that sees this)
-                    if (idx == cnt - 1) umma_commit(qt_free);              // the segment's last read of its queries
+                    if (idx == cnt - 1) umma_commit(q_empty(mt->qsel));   // the segment's last read of its queries
                 }
                 __syncwarp();
             }
@@ -472,7 +477,6 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         const int j = row >> 3, head = row & 7;                  // sibling, head of this row
         const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t o_mine = lane_base + kTmemO + g * kD, o_other = lane_base + kTmemO + (g ^ 1) * kD;
-        const int sw = row & 7;
         const float sc = p.scale_log2e;
         const bool sc_neg = sc < 0.f;
         // The scale used for a row's probabilities is 2^-m_ref, where m_ref trails the true running
@@ -481,7 +485,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         // the maximum by more than that -- a handful of times per segment instead of per tile.
         constexpr float kSlack = 8.f;
         float m_ref = -INFINITY, l = 0.f;
-        uint32_t k = 0, segs = 0, qsegs = 0;                     // tiles this group has taken; segments ended / started
+        uint32_t k = 0, segs = 0;                                // tiles this group has taken; segments ended
         bool ok = true;
         int site = 0;
         for (uint32_t it = 0; ok; ++it) {
@@ -490,32 +494,6 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             if (mt.n == 0) break;
             const bool warp_live = (warp & 3) * 4 < mt.n;        // this warp holds rows of a sharing sibling
             const bool mine = (int)(it & 1u) == g;
-            if (g == 0 && mt.idx == 0) {
-                // ---- a segment starts: group A moves its queries from the staging buffer to TMEM
-                //      (row r of both 64-dim halves -> 64 columns of packed bf16 in lane r)
-                if (!mbar_wait(q_full(mt.qsel), (qsegs >> 1) & 1u, abort_flag)) { ok = false; site = 44; break; }
-                if (qsegs > 0) {
-                    if (!mbar_wait(qt_free, (qsegs - 1) & 1u, abort_flag)) { ok = false; site = 45; break; }
-                    tc_fence_after_sync();
-                }
-                const uint8_t* qsrc = smem + SM::kQOff + mt.qsel * kTQBytes + row * 128;
-                #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t qw[32];
-                    #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        uint4 v = make_uint4(0, 0, 0, 0);
-                        if (row < kTQRows) v = *reinterpret_cast<const uint4*>(qsrc + h * kTQHalfBytes + ((ch ^ sw) << 4));
-                        qw[4 * ch] = v.x; qw[4 * ch + 1] = v.y; qw[4 * ch + 2] = v.z; qw[4 * ch + 3] = v.w;
-                    }
-                    tmem_st32(lane_base + kTmemQ + h * 32, qw);
-                }
-                tmem_wait_st();
-                tc_fence_before_sync();
-                mbar_arrive(q_empty(mt.qsel));                   // the staging buffer may be refilled
-                mbar_arrive(qt_ready);
-                ++qsegs;
-            }
             if (mine) {
                 const bool first = mt.idx < 2;                   // this group's first tile of the segment
                 if (!mbar_wait(s_full(g), k & 1u, abort_flag)) { ok = false; site = 38; break; }
