@@ -27,7 +27,7 @@
 // One softmax warp per SM sub-partition is a serial chain (TMEM load, maximum, 64 exponentials
 // at 4 per clock, pack, store, fences) of about 1,900 clocks per tile, which is below the HBM
 // rate.  So there are TWO softmax warpgroups that take alternate tiles, each with its own
-// score buffer, P columns and O accumulator (TMEM columns: S_A, S_B, P_A, P_B, O_A, O_B); while one group
+// P columns and O accumulator (TMEM columns: three score buffers, P_A, P_B, O_A, O_B); while one group
 // is in its exponentials the other loads its scores.  At the end of a segment the two
 // (m, l, O) states of every row are merged by their log-sum-exp, each group writing half of
 // the output columns.
@@ -41,9 +41,9 @@
 // owns the TMEM allocation, warp 10 issues the P.V MMAs.  One issuing thread for both was the
 // bottleneck (about 90 clocks per tcgen05.mma and as much again in barrier waits and commits,
 // all serial); the two products depend on different events (K landed and score buffer read,
-// against P written and V landed), so each gets its own thread.  Q.K^T of tile i is issued
-// as soon as the score buffer of tile i - 2 has been read, so a group's next scores are ready
-// when it finishes a tile.
+// against P written and V landed), so each gets its own thread.  Tile i's scores go to score buffer
+// i % 3, so Q.K^T of tile i is issued as soon as the scores of tile i - 3 (the other group's) have
+// been read: a group's next scores are computed while it still works on its current tile.
 //
 // Input / output contract is that of the plan: a segment (the part of a unit inside one range)
 // ends with one normalised fp32 partial (out, base-2 lse) per sibling in rows `row .. row + n`
@@ -88,10 +88,11 @@ constexpr int kTPvWarp = 10;                              // issues P.V
 constexpr int kTThreads = 11 * 32;
 constexpr int kTHalfBytes = kTile * 128;                  // 8 KB: 64 tokens x one 64-dim half
 constexpr int kTTileBytes = 2 * kTHalfBytes;              // 16 KB: one K or V tile
-// TMEM columns (512): [0,64) free; S_A [64,128), S_B [128,192); P_A [192,224), P_B [224,256) as
-// packed bf16; O_A [256,384), O_B [384,512)
+// TMEM columns (512): three score buffers S_0 [64,128), S_1 [128,192), S_2 [0,64) used by tile
+// it % 3; P_A [192,224), P_B [224,256) as packed bf16; O_A [256,384), O_B [384,512)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kTmemS = 64, kTmemP = 192, kTmemO = 256;
+constexpr uint32_t kTmemP = 192, kTmemO = 256;
+__host__ __device__ constexpr uint32_t tmem_s_col(uint32_t sb) { return sb == 2 ? 0u : 64u + 64u * sb; }
 
 
 struct TMeta {
@@ -119,8 +120,8 @@ struct TSmem {
     static constexpr int kMetaOff = kXchOff + 2 * kTRows * 8;
     static constexpr int kBarOff = kMetaOff + kTMetaRing * (int)sizeof(TMeta);
     // full_k, empty_k per K stage; full_v, empty_v per V stage; meta_full per record; then pairs:
-    // q_full, q_empty, s_full, s_free, p_full, pv_done; xch_a, xch_b
-    static constexpr int kNumBars = 2 * kTKStages + 2 * kTVStages + kTMetaRing + 14;
+    // pairs q_full, q_empty, p_full, pv_done; xch_a, xch_b; triples s_full, s_free
+    static constexpr int kNumBars = 2 * kTKStages + 2 * kTVStages + kTMetaRing + 20;
     static constexpr int kTmemPtrOff = kBarOff + kNumBars * 8;
     static constexpr int kAbortOff = kTmemPtrOff + 8;
     static constexpr int kTotal = kAbortOff + 8;
@@ -164,8 +165,8 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
     auto meta_full = [&](int s) { return bar_base + 8u * (2 * kTKStages + 2 * kTVStages + s); };
     auto q_full = [&](int i) { return bar_base + 8u * (kB0 + i); };
     auto q_empty = [&](int i) { return bar_base + 8u * (kB0 + 2 + i); };
-    auto s_full = [&](int i) { return bar_base + 8u * (kB0 + 4 + i); };
-    auto s_free = [&](int i) { return bar_base + 8u * (kB0 + 6 + i); };
+    auto s_full = [&](int i) { return bar_base + 8u * (kB0 + 14 + i); };   // per score buffer (3)
+    auto s_free = [&](int i) { return bar_base + 8u * (kB0 + 17 + i); };
     auto p_full = [&](int i) { return bar_base + 8u * (kB0 + 8 + i); };
     auto pv_done = [&](int i) { return bar_base + 8u * (kB0 + 10 + i); };
     const uint32_t xch_a = bar_base + 8u * (kB0 + 12);               // both groups have published (m, l)
@@ -185,11 +186,10 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
         for (int i = 0; i < 2; ++i) {
             mbar_init(q_full(i), 1);
             mbar_init(q_empty(i), 1);                            // one commit after the segment's last Q.K^T
-            mbar_init(s_full(i), 1);
-            mbar_init(s_free(i), 128);
             mbar_init(p_full(i), 128);
             mbar_init(pv_done(i), 1);
         }
+        for (int i = 0; i < 3; ++i) { mbar_init(s_full(i), 1); mbar_init(s_free(i), 128); }
         mbar_init(xch_a, 256);
         mbar_init(xch_b, 256);
         *abort_flag = 0;
@@ -393,7 +393,6 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             int site = 0;
             uint32_t segs = 0;
             for (uint32_t it = 0; ok; ++it) {
-                const int g = it & 1u;
                 const int ks = it % kTKStages;
                 if (!mbar_wait(full_k(ks), (it / kTKStages) & 1u, abort_flag)) { ok = false; site = 43; break; }
                 const TMeta* mt = &meta[it % kTMetaRing];
@@ -403,8 +402,13 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                     if (!mbar_wait(q_full(mt->qsel), (segs >> 1) & 1u, abort_flag)) { ok = false; site = 33; break; }
                     ++segs;
                 }
-                // the group has copied the scores of its previous tile out of the buffer
-                if (!mbar_wait(s_free(g), ((it >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; site = 34; break; }
+                // Three score buffers for two groups: tile `it` uses buffer it % 3, whose previous user
+                // was tile it - 3 of the other group.  So this product does not wait for its own
+                // group to have read the scores of its previous tile (it - 2): those sit in another
+                // buffer, and a group's next scores are computed while it still works on the current
+                // ones, however late it started on them.
+                const uint32_t sb = it % 3u;
+                if (!mbar_wait(s_free(sb), ((it / 3u) & 1u) ^ 1u, abort_flag)) { ok = false; site = 34; break; }
                 tc_fence_after_sync();
                 const uint32_t k_addr = smem_base + ks * kTTileBytes;
                 const uint32_t q_addr = smem_base + SM::kQOff + mt->qsel * kTQBytes;
@@ -414,9 +418,9 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                         const uint32_t koff = (uint32_t)(k16 & 3) * 32u;
                         const uint64_t a = umma_smem_desc(q_addr + (k16 >> 2) * kTQHalfBytes + koff, 16, 1024);
                         const uint64_t b = umma_smem_desc(k_addr + (k16 >> 2) * kTHalfBytes + koff, 16, 1024);
-                        umma_ss(tmem_base + kTmemS + g * kTile, a, b, idesc_qk, k16 > 0);
+                        umma_ss(tmem_base + tmem_s_col(sb), a, b, idesc_qk, k16 > 0);
                     }
-                    umma_commit(s_full(g));       // (the K stage is released by the softmax group that sees this)
+                    umma_commit(s_full(sb));       // (the K stage is released by the softmax group that sees this)
                     if (idx == cnt - 1) umma_commit(q_empty(mt->qsel));   // the segment's last read of its queries
                 }
                 __syncwarp();
@@ -496,7 +500,8 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             const bool mine = (int)(it & 1u) == g;
             if (mine) {
                 const bool first = mt.idx < 2;                   // this group's first tile of the segment
-                if (!mbar_wait(s_full(g), k & 1u, abort_flag)) { ok = false; site = 38; break; }
+                const uint32_t sb = it % 3u;                     // the score buffer of this tile
+                if (!mbar_wait(s_full(sb), (it / 3u) & 1u, abort_flag)) { ok = false; site = 38; break; }
                 // Q.K^T of this tile is complete, so its K stage may be overwritten.  The release is a
                 // plain arrival from a thread that learns of the completion anyway: a second
                 // tcgen05.commit would cost the issuing thread about as much as an MMA.
@@ -507,11 +512,11 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                 bool need = false;
                 if (warp_live) {
                     uint32_t raw[2][32];
-                    tmem_ld32(lane_base + kTmemS + g * kTile, raw[0]);
-                    tmem_ld32(lane_base + kTmemS + g * kTile + 32, raw[1]);
+                    tmem_ld32(lane_base + tmem_s_col(sb), raw[0]);
+                    tmem_ld32(lane_base + tmem_s_col(sb) + 32, raw[1]);
                     tmem_wait_ld();
                     tc_fence_before_sync();
-                    mbar_arrive(s_free(g));
+                    mbar_arrive(s_free(sb));
                     float scl = sc;                              // what the values in raw[] still have to be multiplied by
                     bool neg = sc_neg;
                     if (kPrefill && mt.diag + j < kTile - 1) {
@@ -562,7 +567,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                     sum += sum1;
                 } else {
                     tc_fence_before_sync();
-                    mbar_arrive(s_free(g));
+                    mbar_arrive(s_free(sb));
                 }
                 // this group's previous P.V must be complete before its P tile is overwritten and
                 // before a rescale touches O; the probabilities above were computed while it ran
