@@ -43,8 +43,8 @@ MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074874e9 + 4.741888e6) / 262144
 # The same two counters of one attn_tc_kernel launch on exactly these workloads (profiles/attn_tc_*.md); None for
 # any other workload, and to be removed whenever that kernel changes until the counters are taken again.
 ATTN_TC_TRAFFIC_BYTES = {
-    ("casc_16x10_pre16384_p64", "tcgen05"): 1.080155e9 + 11.060992e6,
-    ("prefill_16x2048_p64", "tcgen05"): 671.256320e6 + 506.075904e6,
+    ("casc_16x10_pre16384_p64", "tcgen05"): 1.080627e9 + 10.573312e6,
+    ("prefill_16x2048_p64", "tcgen05"): 671.279872e6 + 505.919488e6,
 }
 
 
