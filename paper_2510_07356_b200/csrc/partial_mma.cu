@@ -618,31 +618,48 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 if (lane == 0) wait_failed(p, abort_flag, 4);
                 return;
             }
-            const int d = tid;                        // 128 consumer threads = 128 dims
-            #pragma unroll
-            for (int h = 0; h < kGroup; ++h) {
+            // 128 consumer threads = 8 heads x 16 threads; a thread owns dims 4j .. 4j+3 and 64+4j .. 64+4j+3
+            // of one head (16-byte pieces: conflict-free shared-memory reads, 8- or 16-byte stores), so
+            // the head's weights are computed once per thread instead of once per (thread, head)
+            {
+                const int h = tid >> 4, j4 = (tid & 15) * 4;
+                float2 ml[kConsumerWarps];
                 float M = ninf;
                 #pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_ml[(w * kGroup + h) * 2]);
-                float L = 0.f, acc = 0.f;
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    ml[w] = *reinterpret_cast<const float2*>(merge_ml + (w * kGroup + h) * 2);
+                    M = fmaxf(M, ml[w].x);
+                }
+                float L = 0.f;
+                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
                 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float wt = fast_exp2(merge_ml[(w * kGroup + h) * 2] - M);
-                    L = fmaf(merge_ml[(w * kGroup + h) * 2 + 1], wt, L);
-                    acc = fmaf(merge_o[(w * kGroup + h) * kMergeStride + d], wt, acc);
+                    const float wt = fast_exp2(ml[w].x - M);
+                    L = fmaf(ml[w].y, wt, L);
+                    const float* src = merge_o + (w * kGroup + h) * kMergeStride + j4;
+                    const float4 a = *reinterpret_cast<const float4*>(src);
+                    const float4 c = *reinterpret_cast<const float4*>(src + 64);
+                    lo.x = fmaf(a.x, wt, lo.x); lo.y = fmaf(a.y, wt, lo.y); lo.z = fmaf(a.z, wt, lo.z); lo.w = fmaf(a.w, wt, lo.w);
+                    hi.x = fmaf(c.x, wt, hi.x); hi.y = fmaf(c.y, wt, hi.y); hi.z = fmaf(c.z, wt, hi.z); hi.w = fmaf(c.w, wt, hi.w);
                 }
-                const float res = acc / L;
+                const float inv = 1.f / L;
+                lo.x *= inv; lo.y *= inv; lo.z *= inv; lo.w *= inv;
+                hi.x *= inv; hi.y *= inv; hi.z *= inv; hi.w *= inv;
                 const float lse2 = M + log2f(L);
                 if (mt.slot < 0) {
                     if (h < p.group) {
                         const int64_t row = (int64_t)mt.b * p.hq + mt.g * p.group + h;
-                        p.out[row * kD + d] = __float2bfloat16_rn(res);
-                        if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
+                        __nv_bfloat16* dst = p.out + row * kD + j4;
+                        *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w));
+                        *reinterpret_cast<uint2*>(dst + 64) = make_uint2(pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
+                        if (j4 == 0) p.lse[row] = lse2 * 0.6931471805599453f;
                     }
                 } else {
                     const int64_t row = (int64_t)mt.slot * kGroup + h;
-                    p.part_o[row * kD + d] = res;
-                    if (d == 0) p.part_lse[row] = lse2;
+                    float* dst = p.part_o + row * kD + j4;
+                    *reinterpret_cast<float4*>(dst) = lo;
+                    *reinterpret_cast<float4*>(dst + 64) = hi;
+                    if (j4 == 0) p.part_lse[row] = lse2;
                 }
             }
             mbar_arrive(merge_bar1);
