@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one partial_mma_kernel launch divided by its KV tokens, from
 # the ncu capture summarised in profiles/partial_mma_cfg3q_b16_ctx16384.md (page size 64, fused combine, one
 # range per CTA).  Set to None whenever that kernel changes until the counters are taken again.
-MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074874e9 + 4.741888e6) / 262144
+MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074885e9 + 4.496384e6) / 262144
 # The same two counters of one attn_tc_kernel launch on exactly these workloads (profiles/attn_tc_*.md); None for
 # any other workload, and to be removed whenever that kernel changes until the counters are taken again.
 ATTN_TC_TRAFFIC_BYTES = {
