@@ -14,7 +14,9 @@ step with all inputs resident in HBM; `e2e` is the same through the host-buffer 
 with every host<->device copy inside the timed region; `roofline` times the partial kernel
 alone with events the library records around it; `cpu_baseline` is the fp64 CPU oracle on a
 bounded sample of the same workload, and `parity` compares the library's rows of those sampled
-sequences with the oracle's (one-GPU runs only).
+sequences with the oracle's (one-GPU runs only); `sustained` repeats the step (and the read-only
+stream yardstick) back to back for two seconds with the clocks sampled, because a burst of 30 steps and
+a long run can differ under the power cap.
 """
 from __future__ import annotations
 
@@ -63,6 +65,8 @@ def parse_args():
     ap.add_argument("--ranges-per-cta", type=int, default=0)
     ap.add_argument("--min-range-tiles", type=int, default=0)
     ap.add_argument("--num-ranges", type=int, default=0)
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="large workloads: also run the step back to back for this long (0 = skip)")
     ap.add_argument("--loop-steps", type=int, default=16, help="append+attention steps replayed from a CUDA graph")
     ap.add_argument("--fuse-combine", type=int, default=-1)
     ap.add_argument("--claim-ahead", type=int, default=-1)
@@ -788,6 +792,47 @@ def main():
         assert torch.equal(hout.view(torch.int16), out.cpu().view(torch.int16)), "host path differs from device path"
         del hq, hk, hv
 
+    # ---- the same step back to back for about two seconds: what the power cap leaves of the burst figure
+    sustained = None
+    if flush_buf is None and args.sustained_seconds > 0:
+        def back_to_back(fn, one_ms, seconds):
+            chunk = max(10, int(0.1 / max(one_ms * 1e-3, 1e-6)))           # about 0.1 s of calls per event pair
+            marks, t_end = [], time.time() + seconds
+            while time.time() < t_end:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(chunk):
+                    fn()
+                e1.record(stream)
+                e1.synchronize()
+                marks.append(e0.elapsed_time(e1) / chunk)
+            tail = marks[len(marks) // 2:]                                 # the second half: clocks have settled
+            return sum(tail) / len(tail), marks[0], chunk * len(marks)
+
+        sampler2 = ClockSampler(gpu_id)
+        if rank == 0:
+            sampler2.start()
+            time.sleep(0.2)
+        t_s0 = time.time()
+        sus_ms, first_ms, n_steps = back_to_back(step, ms_per_step, args.sustained_seconds)
+        t_s1 = time.time()
+        sus_clocks = sampler2.stop(t_s0, t_s1) if rank == 0 else None
+        sus_ms = over_ranks([sus_ms], "max", dev)[0]
+        sustained = {"ms_per_step": sus_ms, "value": job_bytes / (sus_ms * 1e-3) / 1e9, "unit": UNIT,
+                     "seconds": args.sustained_seconds, "steps": n_steps, "first_chunk_ms_per_step": first_ms,
+                     "clocks": sus_clocks,
+                     "what": "steps back to back; mean of the second half of the interval"}
+        # the read-only stream under the same regime, so that the two can be compared like for like
+        pool_b = w.k_pages.numel() * 2 + w.v_pages.numel() * 2
+        chk_s = torch.zeros(2, dtype=torch.int32, device=dev)
+
+        def probe_s():
+            P.concur_hbm_read_probe(w.k_pages, w.k_pages.numel() * 2, chk_s[0:1], 0, stream.cuda_stream)
+            P.concur_hbm_read_probe(w.v_pages, w.v_pages.numel() * 2, chk_s[1:2], 0, stream.cuda_stream)
+
+        probe_ms, _, _ = back_to_back(probe_s, ms_per_step, args.sustained_seconds / 2)
+        sustained["read_stream_gbs"] = pool_b / (probe_ms * 1e-3) / 1e9
+
     # ---- yardstick: a plain read-only stream over the same two pools (only where they are well above L2)
     read_stream = None
     pool_bytes = w.k_pages.numel() * 2 + w.v_pages.numel() * 2
@@ -866,6 +911,7 @@ def main():
                      "peak_kind": f"of {peak_kind}", "traffic": traffic, "kernel": "partial", "ms": part_ms_avg,
                      "ms_min": min(part_ms)},
         "step_ms_min": min(step_ms), "step_ms_median": statistics.median(step_ms),
+        "sustained": sustained,
         "read_stream": read_stream,
         "frac_of_measured_read_stream": (achieved / read_stream["gbs"]) if read_stream else None,
         "decode_loop": loop, "e2e": e2e, "gpu_launches": (2 if args.kernel == 0 else 3) * K, "clocks": clocks, "device_flags": flags,
