@@ -201,6 +201,9 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr;
+    // everything above (shared-memory set-up, TMEM allocation) overlaps the plan kernel when launched as
+    // its programmatic dependent; the plan's outputs are read only below this wait
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // prefix pass: flat tile space and ranges of the cascade plan; prefill: W = number of units
     const int32_t W = kPrefill ? p.hdr[kHdrTotalTiles] : c.chdr[kHdrTotalTiles];
     const int32_t R = kPrefill ? 0 : c.chdr[kHdrNumRanges];
@@ -704,8 +707,17 @@ cudaError_t launch_attn_tc(const DecodeParams& p, const CascadeParams& c, const 
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<kPrefill>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          TSmem<kPrefill>::kBytes);
     if (e != cudaSuccess) return e;
-    attn_tc_kernel<kPrefill><<<grid, kTThreads, TSmem<kPrefill>::kBytes, stream>>>(p, c, f, mk, mv, mq);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kTThreads);
+    cfg.dynamicSmemBytes = TSmem<kPrefill>::kBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attn_tc_kernel<kPrefill>, p, c, f, mk, mv, mq);
 }
 
 constexpr int kPrefillPlanThreads = 1024;
@@ -722,6 +734,7 @@ __global__ void __launch_bounds__(kPrefillPlanThreads) plan_prefill_kernel(Decod
     __shared__ int32_t warp_sums[kPrefillPlanThreads / 32];
     __shared__ int32_t carry_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the attention kernel's prologue may start
     if (tid == 0) { carry_s = 0; p.tiles_prefix[0] = 0; }
     __syncthreads();
     const int64_t max_len = (int64_t)p.bt_stride * p.page_size;

@@ -53,6 +53,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_cascade_kernel(DecodeParams
     const int lane = tid & 31, warp = tid >> 5;
     const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
     uint32_t flags = 0;
+    // the prefix-pass kernel is launched as this grid's programmatic dependent: its prologue may start now,
+    // it waits for this grid to finish before it reads the plan
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- per group: shared tiles, and each member's offset / group id
     if (tid == 0) { carry = 0; c.ptiles_prefix[0] = 0; }
