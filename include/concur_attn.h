@@ -62,6 +62,8 @@ typedef enum {
 #define CONCUR_FLAG_BAD_PAGE_ID 1u  /* a used block-table entry was outside [0, num_pages): clamped    */
 #define CONCUR_FLAG_BAD_SEQ_LEN 2u  /* a seq_lens entry was outside [0, stride*P]: clamped             */
 #define CONCUR_FLAG_WAIT_LIMIT  4u  /* an in-kernel wait gave up; results of that call are invalid      */
+#define CONCUR_FLAG_BAD_GROUP   8u  /* cascade step: group_start was not 0 <= g[0] <= g[1] <= ... <= batch;
+                                       the call then shared nothing and computed the plain step          */
 
 /* Option keys for concur_attn_set_option (tuning and tests; defaults are chosen per call). */
 #define CONCUR_OPT_KERNEL      1    /* 0 = tensor-core partial kernel (default), 1 = scalar-FMA kernel */
@@ -79,7 +81,7 @@ typedef enum {
 #define CONCUR_OPT_FUSE_COMBINE 8   /* tensor-core kernel: 1 (default) = the CTA that finishes a unit's last
                                        partial merges the unit in-kernel; 0 = separate combine kernel   */
 #define CONCUR_OPT_CLAIM_AHEAD  9   /* tiles before a range's end at which a CTA claims its next range
-                                       (default: at the range's first tile)                              */
+                                       (default: at the range's first tile; 0 = when the range is done) */
 
 #define CONCUR_OPT_PREFIX_KERNEL 10 /* shared-prefix pass of the cascade step: 0 (default) = tcgen05 kernel with
                                        TMEM accumulators, 1 = warp-level mma.sync kernel                 */
@@ -169,7 +171,9 @@ int concur_decode_attn(concur_attn_t* handle,
  * tiles are shared (the rest of the prefix is read per sequence), a group's sequences
  * beyond the tenth read everything themselves, and a prefix longer than the group's
  * shortest sequence is cut to it and recorded as CONCUR_FLAG_BAD_SEQ_LEN.  If the promise
- * is broken the shared part is read through the group's first sequence's table.
+ * is broken the shared part is read through the group's first sequence's table.  A group_start
+ * array that is not non-decreasing within [0, batch] never faults either: the call then shares
+ * nothing, computes what concur_decode_attn computes, and records CONCUR_FLAG_BAD_GROUP.
  *
  * Needs max_batch <= 4096 (CONCUR_ERR_UNSUPPORTED otherwise).  The first cascade call on a
  * handle allocates the cascade workspace (cudaMalloc; CONCUR_ERR_OOM); make it outside any
@@ -291,8 +295,10 @@ int concur_attn_last_plan(concur_attn_t* handle, void* cuda_stream, int32_t* num
  * routine.  Limits: batch <= CONCUR_STATIC_MAX_BATCH (more: CONCUR_ERR_TOO_LARGE, nothing
  * is launched); the plan uses at most CONCUR_STATIC_MAX_RANGES split-KV ranges, so very
  * large batches balance a little more coarsely than through a handle.  Other errors as for
- * concur_decode_attn.  Device-side condition flags (bad page id, bad length) still clamp
- * the access but are not reported by this entry point.
+ * concur_decode_attn.  Device-side conditions are handled as in concur_decode_attn (a bad page
+ * id or length is clamped; a bounded in-kernel wait that gives up ends the kernel, whose results
+ * are then invalid) but this entry point has no handle to report them through: none of the
+ * CONCUR_FLAG_* bits, CONCUR_FLAG_WAIT_LIMIT included, can be read back by its callers.
  *
  * The first call on each device resolves the array's device address
  * (cudaGetSymbolAddress) and reads the SM count; make that first call outside any stream

@@ -21,6 +21,7 @@ CONCUR_ERR_OOM = -5
 CONCUR_FLAG_BAD_PAGE_ID = 1
 CONCUR_FLAG_BAD_SEQ_LEN = 2
 CONCUR_FLAG_WAIT_LIMIT = 4
+CONCUR_FLAG_BAD_GROUP = 8
 
 CONCUR_KV_HEAD_MAJOR = 0
 CONCUR_KV_TOKEN_MAJOR = 1

@@ -296,7 +296,6 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
     c.group_start = group_start;
     c.prefix_lens = prefix_lens;
     c.num_groups = num_groups;
-    c.max_rows = lay.max_rows;
     c.grid_ctas = h->sm_count;
     c.chdr = reinterpret_cast<int32_t*>(cw + lay.chdr);
     c.tok_offset = reinterpret_cast<int32_t*>(cw + lay.tok_offset);

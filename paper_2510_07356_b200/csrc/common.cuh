@@ -18,6 +18,7 @@ constexpr int kRowBytes = kD * 2;
 constexpr uint32_t kFlagBadPage = 1u;
 constexpr uint32_t kFlagBadLen = 2u;
 constexpr uint32_t kFlagWaitLimit = 4u;
+constexpr uint32_t kFlagBadGroup = 8u;
 
 // Workspace header (int32 words).
 enum HeaderWord : int {
@@ -79,15 +80,15 @@ struct CascadeParams {
     const int32_t* group_start;   // [num_groups + 1] first sequence of each group; last entry = batch
     const int32_t* prefix_lens;   // [num_groups] tokens the group's sequences have in common
     int32_t num_groups;
-    int32_t max_rows;             // capacity of pre_o / pre_lse in (sibling, KV head) rows
     int32_t grid_ctas;
     int32_t* chdr;                // [kHdrWords] W', R', claim counter of the prefix pass
     int32_t* tok_offset;          // [batch] shared tokens handled by the prefix pass (0 if none)
     int32_t* seq_group;           // [batch] group of each sequence
     int32_t* ptiles_prefix;       // [num_groups + 1] exclusive prefix of shared tiles per group
     int32_t* unit_rowbase;        // [num_groups * kHkv + 1] first partial row of each prefix unit
-    float* pre_o;                 // [max_rows][kGroup][kD] normalised partials of the prefix pass
-    float* pre_lse;               // [max_rows][kGroup]     their base-2 log-sum-exp
+    float* pre_o;                 // [rows][kGroup][kD] normalised partials of the prefix pass; rows = 8 x max batch
+                                  // + 10 x CTAs: every unit's siblings once, plus once more per range cut
+    float* pre_lse;               // [rows][kGroup]     their base-2 log-sum-exp
 };
 
 // Prefill (several query tokens per sequence, causal).  Device pointer.

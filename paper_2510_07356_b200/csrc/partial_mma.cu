@@ -358,6 +358,14 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                     if (ok) ++it;
                 }
             }
+            // Whatever claim_ahead is, a range never ends without its successor claimed: a CTA that
+            // streamed a range to its end and found no claim condition met (claim_ahead below 1) takes
+            // its ticket here, so the loop always moves on to a range nobody else has.
+            if (ok && !claimed) {
+                see_plan();
+                if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
+                claimed = true;
+            }
             r = __shfl_sync(0xffffffffu, r_next, 0);
         }
         if (lane == 0) {

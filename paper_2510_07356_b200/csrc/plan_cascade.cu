@@ -60,14 +60,25 @@ __global__ void __launch_bounds__(kPlanThreads) plan_cascade_kernel(DecodeParams
     // ---- per group: shared tiles, and each member's offset / group id
     if (tid == 0) { carry = 0; c.ptiles_prefix[0] = 0; }
     for (int b = tid; b < p.batch; b += kPlanThreads) { c.tok_offset[b] = 0; c.seq_group[b] = -1; }
-    __syncthreads();
+    // The group table is device data and may hold anything.  It is usable only if it is a partition
+    // of [0, batch) into consecutive runs: 0 <= group_start[0], group_start[i] <= group_start[i+1],
+    // group_start[num_groups] <= batch.  Then the groups are disjoint, a group's sharing siblings are
+    // real sequences, and the prefix pass writes at most 8 * batch + 10 * (ranges - 1) partial rows,
+    // which is what the workspace holds.  Any violation turns sharing off for the whole call (every
+    // sequence reads all of its tokens itself: the plain step's result) and is flagged; the later
+    // kernels read group_start only for groups that share tiles, i.e. never in that case.
+    int bad = 0;
+    for (int i = tid; i < c.num_groups; i += kPlanThreads) {
+        const int32_t b0 = c.group_start[i], b1 = c.group_start[i + 1];
+        bad |= (b0 < 0) | (b0 > b1) | (b1 > p.batch);
+    }
+    const bool groups_ok = __syncthreads_or(bad) == 0;
+    if (!groups_ok) flags |= kFlagBadGroup;
     for (int base = 0; base < c.num_groups; base += kPlanThreads) {
         const int i = base + tid;
         int32_t tiles = 0;
-        if (i < c.num_groups) {
-            int32_t b0 = c.group_start[i], b1 = c.group_start[i + 1];
-            if (b0 < 0) b0 = 0;
-            if (b1 > p.batch) b1 = p.batch;
+        if (groups_ok && i < c.num_groups) {
+            const int32_t b0 = c.group_start[i], b1 = c.group_start[i + 1];
             const int32_t n_share = min(b1 - b0, kMaxShare);
             int64_t shared = c.prefix_lens[i];
             if (shared < 0) { shared = 0; flags |= kFlagBadLen; }

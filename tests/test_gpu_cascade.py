@@ -101,6 +101,53 @@ def test_long_shared_prefix_split_over_many_ctas(P):
     attn.close()
 
 
+@pytest.mark.parametrize("prefix_kernel", [0, 1])
+def test_malformed_group_tables_share_nothing_and_are_flagged(P, prefix_kernel):
+    # group_start is device data: whatever it holds, the step must not fault.  A table that is not a
+    # non-decreasing walk through [0, batch] switches sharing off for the call -- the result is the
+    # plain step's -- and sets CONCUR_FLAG_BAD_GROUP.
+    cw = synth.make_cascade_workload("casc_badgroups", GROUPS, 64, 4400, "cuda:0")
+    w = cw.w
+    B_ = w.spec.batch
+    ref_out, ref_lse = oracle_sequences(synth.gather_sequences(w, range(B_)))
+    good = cw.group_start.cpu().tolist()
+    G = len(good) - 1
+    bad_tables = [
+        [0, 10, 1, 11, 2, 12, 3, 13, 4][:G + 1],               # overlapping, non-monotonic
+        [good[0]] + [B_ + 5] * G,                              # beyond the batch
+        [-3] + good[1:],                                       # negative start
+        list(reversed(good)),                                  # decreasing
+        [0] + [2 ** 30] * (G - 1) + [B_],                      # huge entries in the middle
+    ]
+    for table in bad_tables:
+        assert len(table) == G + 1
+        gs = torch.tensor(table, dtype=torch.int32, device="cuda:0")
+        attn = P.DecodeAttention(64, B_, w.block_table.shape[1], 0)
+        attn.set_option(P.CONCUR_OPT_PREFIX_KERNEL, prefix_kernel)
+        out = torch.full_like(w.q, 7.0)
+        lse = torch.full((B_, 64), 7.0, dtype=torch.float32, device="cuda:0")
+        P.concur_decode_attn_cascade(attn.handle, w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, gs,
+                                     cw.prefix_lens, w.scale, out, lse, B_, G, w.num_pages,
+                                     w.block_table.shape[1], torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert attn.status() & P.CONCUR_FLAG_BAD_GROUP, table
+        assert_parity(out, lse, ref_out, ref_lse, f"group table {table}")
+        attn.close()
+    # a table that stops short of the batch is a valid walk: the sequences behind it belong to no group
+    short = torch.tensor(good[:-1] + [good[-1] - 1], dtype=torch.int32, device="cuda:0")
+    attn = P.DecodeAttention(64, B_, w.block_table.shape[1], 0)
+    attn.set_option(P.CONCUR_OPT_PREFIX_KERNEL, prefix_kernel)
+    out = torch.full_like(w.q, 7.0)
+    lse = torch.full((B_, 64), 7.0, dtype=torch.float32, device="cuda:0")
+    P.concur_decode_attn_cascade(attn.handle, w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, short,
+                                 cw.prefix_lens, w.scale, out, lse, B_, G, w.num_pages, w.block_table.shape[1],
+                                 torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert_parity(out, lse, ref_out, ref_lse, "group table one short of the batch")
+    attn.close()
+
+
 def test_cascade_argument_errors(P):
     B = P.binding
     cw = synth.make_cascade_workload("casc_args", [(64, [1, 2])], 16, 4300, "cuda:0")

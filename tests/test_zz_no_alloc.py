@@ -1,6 +1,6 @@
 """The handle-free entry point for callers that cannot allocate device memory
-(concur_decode_attn_static): same results as the regular entry point, on two calls in a
-row that share its built-in workspace.
+(concur_decode_attn_static): the oracle's results, the regular entry point's results, on
+calls in a row that share its built-in workspace, and no change in the device's free memory.
 
 Collected last on purpose: should this addition ever fail, a run that stops at the first
 failure has already executed every other test.
@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import synth
+from helpers import assert_parity, oracle_sequences
 
 pytestmark = pytest.mark.gpu
 
@@ -17,17 +18,20 @@ pytestmark = pytest.mark.gpu
 OUT_ATOL, OUT_RTOL, LSE_ATOL = 4e-3, 1.6e-2, 1e-3
 
 
-def test_static_entry_matches_handle_entry_twice_in_a_row():
+def test_static_entry_matches_oracle_and_handle_entry_twice_in_a_row():
     import __graft_entry__
     __graft_entry__.build()
     import paper_2510_07356_b200 as P
 
     stream = torch.cuda.current_stream().cuda_stream
-    # two different batches, the second one larger, so that anything the first call left in
-    # the shared array would be noticed
+    # different batches one after the other, so that anything an earlier call left in the shared
+    # array would be noticed; the fourth has more sequences than the kernel's shared-memory plan
+    # tables hold (511), so its plan is read from the built-in array itself
+    many = [1 + (37 * i) % 150 for i in range(600)]
     specs = [synth.tiny_spec("na0", (3000, 1, 0, 64, 777, 12000), 64, 501),
              synth.tiny_spec("na1", (9000, 20000, 130, 64, 5, 0, 4100, 2500), 64, 502),
-             synth.tiny_spec("na2", (700, 17, 0, 3000, 33), 16, 503)]
+             synth.tiny_spec("na2", (700, 17, 0, 3000, 33), 16, 503),
+             synth.tiny_spec("na3", many, 16, 504)]
     for spec in specs:
         w = synth.make_workload(spec, "cuda:0")
         B = spec.batch
@@ -35,11 +39,24 @@ def test_static_entry_matches_handle_entry_twice_in_a_row():
         out_ref, lse_ref = ref(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
         out = torch.full_like(w.q, 7.0)
         lse = torch.full((B, 64), 7.0, dtype=torch.float32, device="cuda:0")
-        P.concur_decode_attn_static(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale,
-                                    out, lse, B, w.num_pages, w.block_table.shape[1], spec.page_size, stream)
+
+        def call():
+            P.concur_decode_attn_static(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale,
+                                        out, lse, B, w.num_pages, w.block_table.shape[1], spec.page_size, stream)
+
+        call()                                   # (the very first call also resolves the array's address)
         torch.cuda.synchronize()
+        # the promise in the entry point's name: a call takes no device memory and gives none back
+        free_before = torch.cuda.mem_get_info(0)[0]
+        out.fill_(7.0); lse.fill_(7.0)
+        call()
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info(0)[0] == free_before
+        # against the CPU oracle, element by element ...
+        ref_o, ref_l = oracle_sequences(synth.gather_sequences(w, range(B)))
+        assert_parity(out, lse, ref_o, ref_l, f"static entry, {spec.name}")
+        # ... and against the entry point that owns a workspace
         a, b = out.float(), out_ref.float()
-        assert torch.isfinite(a).all()
         assert ((a - b).abs() <= OUT_ATOL + OUT_RTOL * b.abs()).all()
         empty = torch.isneginf(lse_ref)
         assert torch.equal(torch.isneginf(lse), empty)
