@@ -97,8 +97,10 @@ typedef enum {
 typedef struct concur_attn concur_attn_t;   /* opaque; owns its workspace and nothing else */
 
 typedef struct {
-    int32_t num_q_heads;        /* Hq; supported: 8, 16, ... 64 (group size Hq/Hkv = 1 .. 8), e.g. 64 or 40 */
-    int32_t num_kv_heads;       /* Hkv; supported: 8                                            */
+    int32_t num_q_heads;        /* Hq; supported: Hkv x (1 .. 8), e.g. 64 or 40 over 8 KV heads          */
+    int32_t num_kv_heads;       /* Hkv; supported: 1 .. 8.  A rank of a model that is tensor-parallel over
+                                   its KV heads passes the heads it holds: 8 query over 1 KV head at
+                                   8 ranks of the 64 / 8 geometry, with its own slice of every page     */
     int32_t head_dim;           /* D; supported: 128                                            */
     int32_t page_size;          /* P; supported: 16, 32, 64, 128 tokens                         */
     int32_t max_batch;          /* largest `batch` any call will pass (1 .. 65536)              */

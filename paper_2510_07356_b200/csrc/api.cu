@@ -39,13 +39,16 @@ int check_config(const concur_attn_config_t* c) {
         return CONCUR_ERR_INVALID_ARG;
     if (c->max_batch < 1 || c->max_batch > kMaxBatchLimit) return CONCUR_ERR_INVALID_ARG;
     if (c->max_pages_per_seq < 1) return CONCUR_ERR_INVALID_ARG;
-    if (c->num_kv_heads != kHkv || c->head_dim != kD) return CONCUR_ERR_UNSUPPORTED;
-    if (c->num_q_heads < kHkv || c->num_q_heads > kHq || c->num_q_heads % kHkv != 0) return CONCUR_ERR_UNSUPPORTED;
+    if (c->num_kv_heads < 1 || c->num_kv_heads > kHkv || c->head_dim != kD) return CONCUR_ERR_UNSUPPORTED;
+    // 1 to 8 query heads per KV head
+    if (c->num_q_heads < c->num_kv_heads || c->num_q_heads > kGroup * c->num_kv_heads ||
+        c->num_q_heads % c->num_kv_heads != 0)
+        return CONCUR_ERR_UNSUPPORTED;
     if (c->page_size != 16 && c->page_size != 32 && c->page_size != 64 && c->page_size != 128)
         return CONCUR_ERR_UNSUPPORTED;
     // the flat tile index space must fit int32
     const int64_t tiles_per_seq = ((int64_t)c->max_pages_per_seq * c->page_size + kTile - 1) / kTile;
-    if (tiles_per_seq * c->max_batch * kHkv >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
+    if (tiles_per_seq * c->max_batch * c->num_kv_heads >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
     return CONCUR_OK;
 }
 
@@ -156,8 +159,9 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.box_shift = p.page_shift < 6 ? p.page_shift : 6;
     p.lane_copy = p.box_rows < kTile ? h->small_page_copy : 0;
     p.token_major = h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0;
+    p.hkv = h->cfg.num_kv_heads;
     p.hq = h->cfg.num_q_heads;
-    p.group = h->cfg.num_q_heads / kHkv;
+    p.group = h->cfg.num_q_heads / h->cfg.num_kv_heads;
     const int per_sm = h->kernel == 1 ? partial_scalar_ctas_per_sm() : 1;
     p.grid_ctas = h->grid_ctas > 0 ? h->grid_ctas : h->sm_count * per_sm;
     p.forced_ranges = h->forced_ranges;
@@ -184,7 +188,7 @@ static int check_call(concur_attn_t* h, const void* q, const void* k_pages, cons
     if (batch < 0 || num_pages < 1 || stride < 1) return CONCUR_ERR_INVALID_ARG;
     if (batch > h->cfg.max_batch || stride > h->cfg.max_pages_per_seq) return CONCUR_ERR_TOO_LARGE;
     // pool rows are addressed with int32 coordinates
-    if ((int64_t)num_pages * kHkv * h->cfg.page_size >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
+    if ((int64_t)num_pages * h->cfg.num_kv_heads * h->cfg.page_size >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
     if (batch == 0) return CONCUR_OK;
     if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out || !lse) return CONCUR_ERR_INVALID_ARG;
     if (!aligned(q, ptr_align) || !aligned(k_pages, ptr_align) || !aligned(v_pages, ptr_align) ||
@@ -226,7 +230,7 @@ int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, voi
     if (!h) return CONCUR_ERR_INVALID_ARG;
     if (batch < 0 || num_pages < 1 || block_table_stride < 1) return CONCUR_ERR_INVALID_ARG;
     if (batch > h->cfg.max_batch || block_table_stride > h->cfg.max_pages_per_seq) return CONCUR_ERR_TOO_LARGE;
-    if ((int64_t)num_pages * kHkv * h->cfg.page_size >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
+    if ((int64_t)num_pages * h->cfg.num_kv_heads * h->cfg.page_size >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
     if (batch == 0) return CONCUR_OK;
     if (!k_new || !v_new || !k_pages || !v_pages || !block_table || !seq_lens) return CONCUR_ERR_INVALID_ARG;
     if (!aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(k_pages, 16) || !aligned(v_pages, 16) ||
@@ -238,7 +242,7 @@ int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, voi
     const int32_t shift = P == 16 ? 4 : (P == 32 ? 5 : (P == 64 ? 6 : 7));
     if (launch_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
                       reinterpret_cast<int32_t*>(h->ws + h->lay.hdr), batch, num_pages, block_table_stride, P,
-                      shift, h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0,
+                      shift, h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0, h->cfg.num_kv_heads,
                       static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return CONCUR_ERR_CUDA;
     return CONCUR_OK;
@@ -369,7 +373,7 @@ int concur_decode_attn_host(concur_attn_t* h, const void* q, const void* k_pages
     if (!guard.ok()) return CONCUR_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t q_bytes = (size_t)batch * h->cfg.num_q_heads * kD * 2;
-    const size_t pool_bytes = (size_t)num_pages * kHkv * h->cfg.page_size * kD * 2;
+    const size_t pool_bytes = (size_t)num_pages * h->cfg.num_kv_heads * h->cfg.page_size * kD * 2;
     const size_t bt_bytes = (size_t)batch * block_table_stride * 4;
     const size_t len_bytes = (size_t)batch * 4;
     const size_t lse_bytes = (size_t)batch * h->cfg.num_q_heads * 4;

@@ -5,12 +5,12 @@
 
 namespace concur {
 
-constexpr int kAppendThreads = kHkv * (kRowBytes / 16);    // 8 heads x 16 sixteen-byte pieces
+constexpr int kAppendThreads = kHkv * (kRowBytes / 16);    // up to 8 heads x 16 sixteen-byte pieces
 
 __global__ void __launch_bounds__(kAppendThreads) append_kernel(
         const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* k_pages, uint4* v_pages,
         const int32_t* __restrict__ block_table, int32_t* seq_lens, int32_t* hdr, int32_t num_pages,
-        int32_t bt_stride, int32_t page_size, int32_t page_shift, int32_t token_major) {
+        int32_t bt_stride, int32_t page_size, int32_t page_shift, int32_t token_major, int32_t hkv) {
     const int b = blockIdx.x;
     const int g = threadIdx.x >> 4, piece = threadIdx.x & 15;
     const int64_t pos = seq_lens[b];
@@ -25,22 +25,24 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(
         return;
     }
     const int32_t slot = (int32_t)(pos & (page_size - 1));
-    const int64_t row = token_major ? ((int64_t)page * page_size + slot) * kHkv + g
-                                    : ((int64_t)page * kHkv + g) * page_size + slot;
-    const int64_t src = ((int64_t)b * kHkv + g) * (kRowBytes / 16) + piece;
-    k_pages[row * (kRowBytes / 16) + piece] = k_new[src];
-    v_pages[row * (kRowBytes / 16) + piece] = v_new[src];
+    if (g < hkv) {
+        const int64_t row = token_major ? ((int64_t)page * page_size + slot) * hkv + g
+                                        : ((int64_t)page * hkv + g) * page_size + slot;
+        const int64_t src = ((int64_t)b * hkv + g) * (kRowBytes / 16) + piece;
+        k_pages[row * (kRowBytes / 16) + piece] = k_new[src];
+        v_pages[row * (kRowBytes / 16) + piece] = v_new[src];
+    }
     if (threadIdx.x == 0) seq_lens[b] = (int32_t)pos + 1;
 }
 
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                           const int32_t* block_table, int32_t* seq_lens, int32_t* hdr, int32_t batch,
                           int32_t num_pages, int32_t bt_stride, int32_t page_size, int32_t page_shift,
-                          int32_t token_major, cudaStream_t stream) {
+                          int32_t token_major, int32_t hkv, cudaStream_t stream) {
     append_kernel<<<batch, kAppendThreads, 0, stream>>>(
         static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), static_cast<uint4*>(k_pages),
         static_cast<uint4*>(v_pages), block_table, seq_lens, hdr, num_pages, bt_stride, page_size, page_shift,
-        token_major);
+        token_major, hkv);
     return cudaGetLastError();
 }
 

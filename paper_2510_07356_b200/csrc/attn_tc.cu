@@ -322,9 +322,9 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                 int32_t x = x0;
                 while (ok && x < x1) {
                     // the prefix unit (group i, KV head g) that holds flat tile x
-                    const int32_t i = find_sequence(c.ptiles_prefix, c.num_groups, x);
+                    const int32_t i = find_sequence(c.ptiles_prefix, c.num_groups, x, p.hkv);
                     const int32_t t_i = c.ptiles_prefix[i + 1] - c.ptiles_prefix[i];
-                    const int32_t base = kHkv * c.ptiles_prefix[i];
+                    const int32_t base = p.hkv * c.ptiles_prefix[i];
                     const int32_t g = (x - base) / t_i;
                     const int32_t unit_start = base + g * t_i;
                     const int32_t tile0 = x - unit_start;
@@ -333,7 +333,7 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                     const int32_t b0 = c.group_start[i];
                     const int32_t n = min(c.group_start[i + 1] - b0, kMaxShare);
                     const int32_t split = r - range_of(W, R, unit_start);
-                    const int32_t row = c.unit_rowbase[i * kHkv + g] + split * n;
+                    const int32_t row = c.unit_rowbase[i * p.hkv + g] + split * n;
                     // shared tiles are whole; they are read through the first sibling's table row
                     stream_segment(p.block_table + (int64_t)b0 * p.bt_stride, g, tile0, tile1, n, row, b0,
                                    1 << 28, tile1 * kTile - 1);
@@ -347,10 +347,10 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
             while (ok && r < W) {
                 int32_t r_next = 0;
                 if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
-                const int32_t b = find_sequence(p.tiles_prefix, p.batch, r);
-                const int32_t local = r - kHkv * p.tiles_prefix[b];
+                const int32_t b = find_sequence(p.tiles_prefix, p.batch, r, p.hkv);
+                const int32_t local = r - p.hkv * p.tiles_prefix[b];
                 const int32_t nqb = p.tiles_prefix[b + 1] - p.tiles_prefix[b];
-                const int32_t qb = nqb - 1 - local / kHkv, g = local % kHkv;
+                const int32_t qb = nqb - 1 - local / p.hkv, g = local % p.hkv;
                 int64_t len = p.seq_lens[b];
                 len = len < 0 ? 0 : (len > max_len ? max_len : len);
                 int32_t q_len = f.q_start[b + 1] - f.q_start[b];
@@ -696,8 +696,8 @@ template <bool kPrefill>
 cudaError_t launch_attn_tc(const DecodeParams& p, const CascadeParams& c, const PrefillParams& f, uint64_t q_rows,
                            int grid, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
-    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
-    const uint32_t planes = p.token_major ? 2 * kHkv : 2;
+    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : p.hkv);
+    const uint32_t planes = p.token_major ? 2 * p.hkv : 2;
     // a 64-token page is a whole tile: both halves come with one copy ([half][row][128 B])
     const uint32_t halves = p.box_rows == kTile ? 2 : 1;
     if (!make_rows_map(&mk, p.k_pages, pool_rows, p.box_rows, halves, planes) ||
@@ -777,8 +777,8 @@ __global__ void __launch_bounds__(kPrefillPlanThreads) plan_prefill_kernel(Decod
     }
     if (flags) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), flags);
     if (tid == 0) {
-        p.hdr[kHdrTotalTiles] = kHkv * carry_s;          // units
-        p.hdr[kHdrNumRanges] = kHkv * carry_s;
+        p.hdr[kHdrTotalTiles] = p.hkv * carry_s;         // units
+        p.hdr[kHdrNumRanges] = p.hkv * carry_s;
         p.hdr[kHdrClaim] = p.grid_ctas;
     }
 }

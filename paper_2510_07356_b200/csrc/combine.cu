@@ -10,7 +10,7 @@ namespace concur {
 constexpr int kCombineThreads = kD;
 
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p) {
-    const int b = blockIdx.x / kHkv, g = blockIdx.x % kHkv;
+    const int b = blockIdx.x / p.hkv, g = blockIdx.x % p.hkv;
     const int d = threadIdx.x;
     const int32_t tiles_b = p.tiles_prefix[b + 1] - p.tiles_prefix[b];
     const int64_t row0 = (int64_t)b * p.hq + g * p.group;
@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
         return;
     }
     const int32_t R = p.hdr[kHdrNumRanges];
-    const int32_t unit_start = kHkv * p.tiles_prefix[b] + g * tiles_b;
+    const int32_t unit_start = p.hkv * p.tiles_prefix[b] + g * tiles_b;
     const int32_t unit_end = unit_start + tiles_b;
     const int32_t r_lo = find_range(p.range_start, R, unit_start);
     const int32_t r_hi = find_range(p.range_start, R, unit_end - 1);
@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
 }
 
 cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream) {
-    combine_kernel<<<p.batch * kHkv, kCombineThreads, 0, stream>>>(p);
+    combine_kernel<<<p.batch * p.hkv, kCombineThreads, 0, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -61,7 +61,7 @@ cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream) {
 namespace concur {
 
 __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(DecodeParams p, CascadeParams c) {
-    const int b = blockIdx.x / kHkv, g = blockIdx.x % kHkv;
+    const int b = blockIdx.x / p.hkv, g = blockIdx.x % p.hkv;
     const int d = threadIdx.x;
     float mx[kGroup], z[kGroup], acc[kGroup];
     #pragma unroll
@@ -83,10 +83,10 @@ __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(Decode
     const int32_t tiles_b = p.tiles_prefix[b + 1] - p.tiles_prefix[b];
     if (tiles_b > 0) {
         const int32_t W = p.hdr[kHdrTotalTiles], R = p.hdr[kHdrNumRanges];
-        const int32_t unit_start = kHkv * p.tiles_prefix[b] + g * tiles_b;
+        const int32_t unit_start = p.hkv * p.tiles_prefix[b] + g * tiles_b;
         const int32_t r_lo = range_of(W, R, unit_start), r_hi = range_of(W, R, unit_start + tiles_b - 1);
         for (int32_t r = r_lo; r <= r_hi; ++r) {
-            const int64_t slot = (int64_t)r + b * kHkv + g;
+            const int64_t slot = (int64_t)r + b * p.hkv + g;
             add(p.part_lse + slot * kGroup, p.part_o + slot * kGroup * kD);
         }
     }
@@ -97,9 +97,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(Decode
         const int32_t b0 = c.group_start[i];
         const int32_t n = min(c.group_start[i + 1] - b0, kMaxShare);
         const int32_t W = c.chdr[kHdrTotalTiles], R = c.chdr[kHdrNumRanges];
-        const int32_t start = kHkv * c.ptiles_prefix[i] + g * t_i;
+        const int32_t start = p.hkv * c.ptiles_prefix[i] + g * t_i;
         const int32_t splits = range_of(W, R, start + t_i - 1) - range_of(W, R, start) + 1;
-        const int64_t row0 = c.unit_rowbase[i * kHkv + g] + (b - b0);
+        const int64_t row0 = c.unit_rowbase[i * p.hkv + g] + (b - b0);
         for (int32_t s = 0; s < splits; ++s) {
             const int64_t row = row0 + (int64_t)s * n;
             add(c.pre_lse + row * kGroup, c.pre_o + row * kGroup * kD);
@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(Decode
 }
 
 cudaError_t launch_combine_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
-    combine_cascade_kernel<<<p.batch * kHkv, kCombineThreads, 0, stream>>>(p, c);
+    combine_cascade_kernel<<<p.batch * p.hkv, kCombineThreads, 0, stream>>>(p, c);
     return cudaGetLastError();
 }
 

@@ -8,8 +8,8 @@
 
 namespace concur {
 
-constexpr int kHq = 64;          // query heads
-constexpr int kHkv = 8;          // KV heads
+constexpr int kHq = 64;          // most query heads
+constexpr int kHkv = 8;          // most KV heads (workspace capacities); a call's count is DecodeParams::hkv
 constexpr int kGroup = 8;        // most query heads per KV head; width of every partial slot
 constexpr int kD = 128;          // head dimension
 constexpr int kTile = 64;        // tokens per KV tile: the unit the plan counts in
@@ -51,7 +51,8 @@ struct DecodeParams {
                               // 16-byte asynchronous copies instead of one TMA box per (page, head) chunk
     int32_t token_major;      // 0: pools are [page][KV head][slot][D]; 1: [page][slot][KV head][D]
     int32_t group;            // query heads per KV head (1..kGroup); heads g*group .. g*group+group-1 share KV head g
-    int32_t hq;               // query heads = kHkv * group
+    int32_t hkv;              // KV heads of the pools and of k_new / v_new: 1, 2, 4 or 8
+    int32_t hq;               // query heads = hkv * group
     // plan controls
     int32_t grid_ctas;        // CTAs the partial kernel is launched with
     int32_t forced_ranges;    // > 0: use exactly this many ranges (clamped to [1, min(W, max_ranges)])
@@ -66,10 +67,10 @@ struct DecodeParams {
     int32_t* range_start;     // [R + 1] boundaries in flat tile space
     float* part_o;            // [2 * max_ranges][kGroup][kD] normalised partial outputs
     float* part_lse;          // [2 * max_ranges][kGroup]     base-2 log-sum-exp of each partial
-    int32_t* unit_done;       // [batch * kHkv] partial segments finished per (sequence, KV head) unit
+    int32_t* unit_done;       // [batch * hkv] partial segments finished per (sequence, KV head) unit
     // shared-prefix (cascade) mode; both unset in the plain path
     const int32_t* tok_offset; // [batch] first token of each sequence that this pass covers (multiple of 64), or null
-    int32_t all_partial;      // 1: every segment writes a partial into slot r + u (u = b * kHkv + g)
+    int32_t all_partial;      // 1: every segment writes a partial into slot r + u (u = b * hkv + g)
 };
 
 constexpr int kMaxShare = 10;     // siblings of a group that share one read of their common prefix
@@ -85,7 +86,7 @@ struct CascadeParams {
     int32_t* tok_offset;          // [batch] shared tokens handled by the prefix pass (0 if none)
     int32_t* seq_group;           // [batch] group of each sequence
     int32_t* ptiles_prefix;       // [num_groups + 1] exclusive prefix of shared tiles per group
-    int32_t* unit_rowbase;        // [num_groups * kHkv + 1] first partial row of each prefix unit
+    int32_t* unit_rowbase;        // [num_groups * hkv + 1] first partial row of each prefix unit
     float* pre_o;                 // [rows][kGroup][kD] normalised partials of the prefix pass; rows = 8 x max batch
                                   // + 10 x CTAs: every unit's siblings once, plus once more per range cut
     float* pre_lse;               // [rows][kGroup]     their base-2 log-sum-exp
@@ -101,12 +102,12 @@ struct PrefillParams {
 // tensor maps over a pool (a row is 64 elements of one half of one 128-wide K or V row; `half` is
 // added to the plane by the caller) and as an element offset for plain loads and stores.
 __device__ __forceinline__ int32_t pool_row(const DecodeParams& p, int32_t page, int32_t g, int32_t slot) {
-    return p.token_major ? page * p.page_size + slot : (page * kHkv + g) * p.page_size + slot;
+    return p.token_major ? page * p.page_size + slot : (page * p.hkv + g) * p.page_size + slot;
 }
 __device__ __forceinline__ int32_t pool_plane(const DecodeParams& p, int32_t g) { return p.token_major ? 2 * g : 0; }
 __device__ __forceinline__ int64_t pool_elem(const DecodeParams& p, int32_t page, int32_t g, int32_t slot) {
-    return p.token_major ? (((int64_t)page * p.page_size + slot) * kHkv + g) * kD
-                         : (((int64_t)page * kHkv + g) * p.page_size + slot) * kD;
+    return p.token_major ? (((int64_t)page * p.page_size + slot) * p.hkv + g) * kD
+                         : (((int64_t)page * p.hkv + g) * p.page_size + slot) * kD;
 }
 
 // Number of split-KV ranges for W flat tiles: as many as keeps every CTA supplied `ranges_per_cta`
@@ -125,7 +126,7 @@ __device__ __forceinline__ int32_t plan_num_ranges(const DecodeParams& p, int32_
         // worth about three tiles; when unit lengths differ much, so do these sums, and a CTA that
         // finishes early then takes a second range off one that does not.  On even batches the
         // second range only costs its start-up.
-        const bool skewed = (int64_t)max_tiles * kHkv * p.batch >= 4 * (int64_t)W;
+        const bool skewed = (int64_t)max_tiles * p.hkv * p.batch >= 4 * (int64_t)W;
         const int32_t per_cta = p.ranges_per_cta > 0 ? p.ranges_per_cta
                                                      : (skewed && W >= p.grid_ctas * 2 * 64 ? 2 : 1);
         const int32_t cap = p.grid_ctas * per_cta;
@@ -150,8 +151,8 @@ __device__ __forceinline__ int32_t range_of(int32_t W, int32_t R, int32_t x) {
     return r;
 }
 
-// The flat tile space lists, for sequence b = 0.., KV head g = 0..7, that unit's tiles:
-// unit (b, g) occupies [kHkv * prefix[b] + g * tiles_b, ... + tiles_b).
+// The flat tile space lists, for sequence b = 0.., KV head g = 0..hkv-1, that unit's tiles:
+// unit (b, g) occupies [hkv * prefix[b] + g * tiles_b, ... + tiles_b).
 struct Segment {
     int32_t b, g;
     int32_t tile0, tile1;     // tiles of the unit covered by this segment, [tile0, tile1)
@@ -159,12 +160,13 @@ struct Segment {
     int32_t slot;             // partial slot, or -1 when the segment covers the whole unit
 };
 
-// Largest b in [0, batch) with kHkv * prefix[b] <= x  (x < W).
-__device__ __forceinline__ int32_t find_sequence(const int32_t* __restrict__ prefix, int32_t batch, int32_t x) {
-    int32_t lo = 0, hi = batch;            // invariant: kHkv*prefix[lo] <= x < kHkv*prefix[hi]
+// Largest b in [0, batch) with hkv * prefix[b] <= x  (x < W).
+__device__ __forceinline__ int32_t find_sequence(const int32_t* __restrict__ prefix, int32_t batch, int32_t x,
+                                                 int32_t hkv) {
+    int32_t lo = 0, hi = batch;            // invariant: hkv*prefix[lo] <= x < hkv*prefix[hi]
     while (hi - lo > 1) {
         int32_t mid = (lo + hi) >> 1;
-        if (kHkv * prefix[mid] <= x) lo = mid; else hi = mid;
+        if (hkv * prefix[mid] <= x) lo = mid; else hi = mid;
     }
     return lo;
 }
@@ -180,12 +182,12 @@ __device__ __forceinline__ int32_t find_range(const int32_t* __restrict__ range_
 }
 
 // Segment of range r that starts at flat tile x (range_start[r] <= x < range_start[r+1]).
-__device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix, int32_t batch,
+__device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix, int32_t batch, int32_t hkv,
                                               int32_t r, int32_t x0, int32_t x1, int32_t x,
                                               int32_t all_partial = 0) {
     Segment s;
-    s.b = find_sequence(prefix, batch, x);
-    int32_t base = kHkv * prefix[s.b];
+    s.b = find_sequence(prefix, batch, x, hkv);
+    int32_t base = hkv * prefix[s.b];
     s.tiles_b = prefix[s.b + 1] - prefix[s.b];
     s.g = (x - base) / s.tiles_b;
     int32_t unit_start = base + s.g * s.tiles_b;
@@ -196,8 +198,8 @@ __device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix
     bool whole = (s.tile0 == 0) && (s.tile1 == s.tiles_b);
     s.slot = whole ? -1 : 2 * r + (x > x0 ? 1 : 0);
     // cascade mode: every segment is a partial; (range, unit) pairs grow strictly along the flat
-    // tile space, so r + u is a unique slot below R + batch * kHkv
-    if (all_partial) s.slot = r + s.b * kHkv + s.g;
+    // tile space, so r + u is a unique slot below R + batch * hkv
+    if (all_partial) s.slot = r + s.b * hkv + s.g;
     return s;
 }
 
@@ -215,6 +217,6 @@ int partial_scalar_ctas_per_sm();
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                           const int32_t* block_table, int32_t* seq_lens, int32_t* hdr, int32_t batch,
                           int32_t num_pages, int32_t bt_stride, int32_t page_size, int32_t page_shift,
-                          int32_t token_major, cudaStream_t stream);
+                          int32_t token_major, int32_t hkv, cudaStream_t stream);
 
 }  // namespace concur

@@ -188,7 +188,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             carry += total;
             __syncthreads();
         }
-        W = kHkv * carry;
+        W = p.hkv * carry;
         R = plan_num_ranges(p, W, longest);
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -219,7 +219,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     auto copy_quarter = [&](int s, int w, int32_t n_valid, int32_t g, int32_t page) {
         const uint32_t hi = lane >> 4, c16 = lane & 15;
         const uint32_t soff = (c16 >> 3) * (uint32_t)P * 128u + hi * 128u + (((c16 & 7u) ^ hi) << 4);
-        const uint32_t row_bytes = p.token_major ? (uint32_t)(kHkv * kRowBytes) : (uint32_t)kRowBytes;
+        const uint32_t row_bytes = p.token_major ? (uint32_t)(p.hkv * kRowBytes) : (uint32_t)kRowBytes;
         const int32_t row0 = 16 * w;                              // first row of the quarter in its tile
         const bool live = row0 < ((n_valid + P - 1) & ~(P - 1));  // whole boxes are read, as the TMA path does
         const int32_t rb = row0 & (P - 1);                        // ... and in its page
@@ -271,7 +271,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             const int32_t x1 = range_begin(W, R, r + 1);
             int32_t x = x0;
             while (ok && x < x1) {
-                const Segment sg = segment_at(prefix, p.batch, r, x0, x1, x, p.all_partial);
+                const Segment sg = segment_at(prefix, p.batch, p.hkv, r, x0, x1, x, p.all_partial);
                 x += sg.tile1 - sg.tile0;
                 int32_t n;                // tokens of the sequence that this pass covers
                 if (cached) n = sm_len[sg.b];
@@ -416,7 +416,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             int32_t ticket = 0;
             if (lane == 0)
                 asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;"
-                             : "=r"(ticket) : "l"(p.unit_done + jb * kHkv + jg), "r"(1) : "memory");
+                             : "=r"(ticket) : "l"(p.unit_done + jb * p.hkv + jg), "r"(1) : "memory");
             ticket = __shfl_sync(0xffffffffu, ticket, 0);
             __syncwarp();
             const int32_t r_lo = range_of(W, R, ju);
@@ -707,8 +707,8 @@ cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
     }
     CUtensorMap map_k, map_v;
     // one box {64, rows of a box, 2} = the part of one (page, KV head) chunk that belongs to a tile
-    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
-    const uint32_t planes = p.token_major ? 2 * kHkv : 2;
+    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : p.hkv);
+    const uint32_t planes = p.token_major ? 2 * p.hkv : 2;
     if (!make_rows_map(&map_k, p.k_pages, pool_rows, p.box_rows, 2, planes) ||
         !make_rows_map(&map_v, p.v_pages, pool_rows, p.box_rows, 2, planes))
         return cudaErrorInvalidValue;

@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
         const int32_t x0 = p.range_start[r], x1 = p.range_start[r + 1];
         int32_t x = x0;
         while (x < x1) {
-            const Segment sg = segment_at(p.tiles_prefix, p.batch, r, x0, x1, x, p.all_partial);
+            const Segment sg = segment_at(p.tiles_prefix, p.batch, p.hkv, r, x0, x1, x, p.all_partial);
             x += sg.tile1 - sg.tile0;
 
             int64_t n = p.seq_lens[sg.b];
@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
                 }
                 const int32_t slot = t & (p.page_size - 1);
                 const int64_t elem = pool_elem(p, page, sg.g, slot);
-                const int64_t tok_stride = p.token_major ? kHkv * (kD / 8) : kD / 8;   // uint4s between consecutive tokens
+                const int64_t tok_stride = p.token_major ? p.hkv * (kD / 8) : kD / 8;   // uint4s between consecutive tokens
                 const uint4* kp = reinterpret_cast<const uint4*>(p.k_pages + elem) + sub;
                 const uint4* vp = reinterpret_cast<const uint4*>(p.v_pages + elem) + sub;
                 uint4 kr[kTokPerStep], vr[kTokPerStep];

@@ -77,10 +77,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
         __syncthreads();
     }
     if (flags) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), flags);
-    for (int i = tid; i < p.batch * kHkv; i += kPlanThreads) p.unit_done[i] = 0;
+    for (int i = tid; i < p.batch * p.hkv; i += kPlanThreads) p.unit_done[i] = 0;
 
     if (tid == 0) {
-        const int32_t W = kHkv * carry_s;
+        const int32_t W = p.hkv * carry_s;
         const int32_t R = plan_num_ranges(p, W, max_s);
         p.hdr[kHdrTotalTiles] = W;
         p.hdr[kHdrNumRanges] = R;
@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
     }
     __syncthreads();
     const int32_t R = ranges_s;
-    const int64_t W = (int64_t)kHkv * carry_s;
+    const int64_t W = (int64_t)p.hkv * carry_s;
     for (int r = tid; r <= R; r += kPlanThreads)
         p.range_start[r] = (R > 0) ? (int32_t)((W * r) / R) : 0;
 }

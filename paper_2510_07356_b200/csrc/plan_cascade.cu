@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_cascade_kernel(DecodeParams
     }
     __syncthreads();
     if (tid == 0) {
-        const int32_t W = kHkv * carry;                  // prefix pass: flat tile space
+        const int32_t W = p.hkv * carry;                 // prefix pass: flat tile space
         int32_t R = W / 2;
         if (R > c.grid_ctas) R = c.grid_ctas;
         if (R < 1 && W > 0) R = 1;
@@ -112,16 +112,16 @@ __global__ void __launch_bounds__(kPlanThreads) plan_cascade_kernel(DecodeParams
 
     // ---- per prefix unit (group, KV head): rows of partials = splits x sharing siblings
     const int32_t Wp = Ws, Rp = Rs;
-    const int32_t units = c.num_groups * kHkv;
+    const int32_t units = c.num_groups * p.hkv;
     if (tid == 0) c.unit_rowbase[0] = 0;
     for (int base = 0; base < units; base += kPlanThreads) {
         const int u = base + tid;
         int32_t rows = 0;
         if (u < units) {
-            const int i = u / kHkv, g = u % kHkv;
+            const int i = u / p.hkv, g = u % p.hkv;
             const int32_t t = c.ptiles_prefix[i + 1] - c.ptiles_prefix[i];
             if (t > 0) {
-                const int32_t start = kHkv * c.ptiles_prefix[i] + g * t;
+                const int32_t start = p.hkv * c.ptiles_prefix[i] + g * t;
                 const int32_t splits = range_of(Wp, Rp, start + t - 1) - range_of(Wp, Rp, start) + 1;
                 const int32_t n_share = min(c.group_start[i + 1] - c.group_start[i], kMaxShare);
                 rows = splits * n_share;
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_cascade_kernel(DecodeParams
     if (flags) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), flags);
     __syncthreads();
     if (tid == 0) {
-        const int32_t W = kHkv * carry;
+        const int32_t W = p.hkv * carry;
         int32_t R = p.forced_ranges > 0 ? p.forced_ranges : min(W / p.min_range_tiles, p.grid_ctas * (p.ranges_per_cta > 0 ? p.ranges_per_cta : 1));
         if (R > p.max_ranges) R = p.max_ranges;
         if (R > W) R = W;

@@ -116,9 +116,9 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
             int32_t x = x0;
             while (ok && x < x1) {
                 // the prefix unit (group i, KV head g) that holds flat tile x
-                const int32_t i = find_sequence(c.ptiles_prefix, c.num_groups, x);
+                const int32_t i = find_sequence(c.ptiles_prefix, c.num_groups, x, p.hkv);
                 const int32_t t_i = c.ptiles_prefix[i + 1] - c.ptiles_prefix[i];
-                const int32_t base = kHkv * c.ptiles_prefix[i];
+                const int32_t base = p.hkv * c.ptiles_prefix[i];
                 const int32_t g = (x - base) / t_i;
                 const int32_t unit_start = base + g * t_i;
                 const int32_t tile0 = x - unit_start;
@@ -127,7 +127,7 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                 const int32_t b0 = c.group_start[i];
                 const int32_t n = min(c.group_start[i + 1] - b0, min(kMaxShare, NS));
                 const int32_t split = r - range_of(W, R, unit_start);
-                const int32_t row = c.unit_rowbase[i * kHkv + g] + split * n;
+                const int32_t row = c.unit_rowbase[i * p.hkv + g] + split * n;
                 const int32_t qsel = seg & 1;
                 const int32_t* table = p.block_table + (int64_t)b0 * p.bt_stride;   // the first sibling's pages
                 const int32_t page_end = (tile1 * kTile + page_mask) >> p.page_shift;
@@ -430,8 +430,8 @@ cudaError_t launch_ns(const DecodeParams& p, const CascadeParams& c, const CUten
 
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream) {
     CUtensorMap mk, mv, mq;
-    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : kHkv);
-    const uint32_t planes = p.token_major ? 2 * kHkv : 2;
+    const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : p.hkv);
+    const uint32_t planes = p.token_major ? 2 * p.hkv : 2;
     if (!make_rows_map(&mk, p.k_pages, pool_rows, p.box_rows, 2, planes) ||
         !make_rows_map(&mv, p.v_pages, pool_rows, p.box_rows, 2, planes) ||
         !make_rows_map(&mq, p.q, (uint64_t)p.batch * p.hq, kGroup, 2))

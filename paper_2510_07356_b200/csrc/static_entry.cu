@@ -107,6 +107,7 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.box_rows = page_size;
     p.box_shift = p.page_shift;
     p.lane_copy = page_size < kTile ? 1 : 0;
+    p.hkv = kHkv;
     p.hq = kHq;
     p.group = kGroup;
     p.grid_ctas = s->sm_count;

@@ -11,12 +11,12 @@ class DecodeAttention:
     torch's current stream and returns (out bf16 [B][Hq][D], lse fp32 [B][Hq])."""
 
     def __init__(self, page_size: int, max_batch: int, max_pages_per_seq: int, device: int = 0,
-                 num_q_heads: int = 64, kv_layout: int = 0):
+                 num_q_heads: int = 64, kv_layout: int = 0, num_kv_heads: int = 8):
         if not torch.cuda.is_available():
             raise RuntimeError("concur_attn needs a CUDA device; there is no CPU path")
         self.device = torch.device("cuda", device)
         self.cfg = B.make_config(page_size, max_batch, max_pages_per_seq, device, num_q_heads=num_q_heads,
-                                 kv_layout=kv_layout)
+                                 num_kv_heads=num_kv_heads, kv_layout=kv_layout)
         self.handle = B.concur_attn_create(self.cfg)
 
     def set_option(self, key: int, value: int):

@@ -210,6 +210,23 @@ def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = Non
         lens_host=lens, table_host=table)
 
 
+def shard_kv_heads(w: Workload, rank: int, world: int) -> Workload:
+    """Rank `rank`'s slice of a workload under tensor parallelism over the KV heads: KV heads
+    [rank * Hkv / world, (rank + 1) * Hkv / world) of every page, and the query heads that attend to
+    them.  Tables and lengths are shared by all ranks.  Slicing only (contiguous copies)."""
+    s = w.spec
+    assert s.num_kv_heads % world == 0 and 0 <= rank < world
+    hkv = s.num_kv_heads // world
+    hq = s.num_q_heads // world
+    from dataclasses import replace
+    spec = replace(s, name=f"{s.name}_kvshard{rank}of{world}", num_q_heads=hq, num_kv_heads=hkv)
+    return Workload(spec=spec, q=w.q[:, rank * hq:(rank + 1) * hq].contiguous(),
+                    k_pages=w.k_pages[:, rank * hkv:(rank + 1) * hkv].contiguous(),
+                    v_pages=w.v_pages[:, rank * hkv:(rank + 1) * hkv].contiguous(),
+                    block_table=w.block_table, seq_lens=w.seq_lens, scale=w.scale,
+                    lens_host=w.lens_host, table_host=w.table_host)
+
+
 def tiny_spec(name, lens, page_size, seed, permute=True, **kw) -> Spec:
     """A small hand-sized workload with the given context lengths."""
     return Spec(name, len(lens), page_size, ("list", list(lens)), permute_pages=permute, seed=seed, **kw)
@@ -268,7 +285,7 @@ class CascadeWorkload:
 
 
 def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0,
-                          num_q_heads=NUM_Q_HEADS) -> CascadeWorkload:
+                          num_q_heads=NUM_Q_HEADS, num_kv_heads=NUM_KV_HEADS) -> CascadeWorkload:
     """groups: list of (shared_tokens, [own_tokens of each sibling]).  `shared_tokens` must be a
     multiple of the page size (only whole pages can be shared physically).  Sequence lengths are
     shared + own; siblings point at the same physical pages for the shared part; all pages are
@@ -282,7 +299,7 @@ def make_cascade_workload(name, groups, page_size, seed, device="cpu", q_std=1.0
         pre.append(shared)
     lens = np.asarray(lens, dtype=np.int32)
     spec = Spec(name, len(lens), P, ("list", [int(x) for x in lens]), seed=seed, q_std=q_std,
-                num_q_heads=num_q_heads)
+                num_q_heads=num_q_heads, num_kv_heads=num_kv_heads)
     # page allocation: shared pages once per group, then each sibling's own pages
     rows, total = [], 0
     for (shared, owns), b0 in zip(groups, gstart[:-1]):
@@ -385,11 +402,12 @@ class PrefillWorkload:
 
 
 def make_prefill_workload(name, lens, q_lens, page_size, seed, device="cpu", num_q_heads=NUM_Q_HEADS,
-                          q_std=1.0) -> PrefillWorkload:
+                          q_std=1.0, num_kv_heads=NUM_KV_HEADS) -> PrefillWorkload:
     """Sequences of `lens` cached tokens whose last `q_lens` tokens are the query tokens
     (q_lens[b] <= lens[b]; q_lens == lens is the prefill of a whole prompt, smaller values a
     chunk of it).  Pools, tables and poisoning as in make_workload; q ~ N(0, q_std^2)."""
-    spec = tiny_spec(name, [int(x) for x in lens], page_size, seed, num_q_heads=num_q_heads, q_std=q_std)
+    spec = tiny_spec(name, [int(x) for x in lens], page_size, seed, num_q_heads=num_q_heads, q_std=q_std,
+                     num_kv_heads=num_kv_heads)
     w = make_workload(spec, device)
     qs = np.zeros(len(lens) + 1, dtype=np.int32)
     qs[1:] = np.cumsum(np.asarray(q_lens, dtype=np.int64))
@@ -415,7 +433,7 @@ def prefill_as_decode(pw: PrefillWorkload, tokens) -> Workload:
     lens = np.asarray(lens, dtype=np.int32)
     table = np.stack(rows).astype(np.int32) if rows else np.zeros((0, w.table_host.shape[1]), np.int32)
     spec = Spec(w.spec.name + "_as_decode", len(lens), w.spec.page_size, ("list", [int(x) for x in lens]),
-                seed=w.spec.seed, num_q_heads=w.spec.num_q_heads)
+                seed=w.spec.seed, num_q_heads=w.spec.num_q_heads, num_kv_heads=w.spec.num_kv_heads)
     idx = torch.as_tensor(tokens, dtype=torch.long)
     return Workload(spec=spec, q=w.q.cpu()[idx], k_pages=w.k_pages.cpu(), v_pages=w.v_pages.cpu(),
                     block_table=torch.from_numpy(table), seq_lens=torch.from_numpy(lens), scale=w.scale,
