@@ -2,6 +2,15 @@
 C ABI on seeded synthetic long-trace workloads.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+                    [--shard replicas|kv-heads]
+
+With --gpus N > 1 and no WORLD_SIZE in the environment the script starts its N ranks itself (one
+process per GPU, rendezvous on 127.0.0.1); under an outside launcher that sets RANK / LOCAL_RANK /
+WORLD_SIZE it is one of the ranks.  Either way the world size must equal N or the run fails.
+--shard replicas (default): every rank decodes its own batch of the workload's shape (weak scaling);
+--shard kv-heads: the ranks split ONE batch the way tensor parallelism does, each holding Hkv / N KV
+heads of every page and the query heads that attend to them (strong scaling, no collective inside
+attention).  NCCL carries only the barrier and the max / sum of the timings.
 
 NAME is one of synth.SPECS (plain decode step; the default is the 64 x 16,384 configuration) or of
 synth.CASCADE_SPECS (shared-prefix step: `value` counts the shared pages once, `logical_gbs` as if
@@ -39,11 +48,11 @@ DEFAULT_WORKLOAD = "cfg3_b64_ctx16384_p64"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one partial_mma_kernel launch divided by its KV tokens, from
-# the ncu capture summarised in profiles/partial_mma_cfg3q_b16_ctx16384.md (page size 64, fused combine, one
-# range per CTA).  Set to None whenever that kernel changes until the counters are taken again.
+# an ncu capture of a quarter of the 64 x 16,384 configuration (page size 64, fused combine, one range per
+# CTA).  Set to None whenever that kernel changes until the counters are taken again.
 MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074885e9 + 4.496384e6) / 262144
-# The same two counters of one attn_tc_kernel launch on exactly these workloads (profiles/attn_tc_*.md); None for
-# any other workload, and to be removed whenever that kernel changes until the counters are taken again.
+# The same two counters of one attn_tc_kernel launch on exactly these workloads; None for any other
+# workload, and to be removed whenever that kernel changes until the counters are taken again.
 ATTN_TC_TRAFFIC_BYTES = {
     ("casc_16x10_pre16384_p64", "tcgen05"): 1.080627e9 + 10.573312e6,
     ("prefill_16x2048_p64", "tcgen05"): 671.279872e6 + 505.919488e6,
@@ -57,6 +66,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "kv-heads"],
+                    help="N > 1: independent batches per rank, or one batch split over the KV heads")
     ap.add_argument("--kernel", type=int, default=0, help="0 tensor-core partial kernel, 1 scalar-FMA")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -260,6 +271,91 @@ def rank_spec(spec, rank: int, world: int):
     return replace(spec, seed=spec.seed + 100 * rank)
 
 
+def rank_workload(spec, rank: int, world: int, shard: str, device, **kw):
+    """What rank `rank` of `world` works on.  replicas: its own batch of the workload's shape (own
+    seed).  kv-heads: the one batch every rank draws identically, cut to this rank's KV heads of
+    every page and the query heads that attend to them."""
+    import synth
+    if shard == "kv-heads" and world > 1:
+        if spec.num_kv_heads % world:
+            raise SystemExit(f"--shard kv-heads: {spec.num_kv_heads} KV heads do not split over {world} ranks")
+        return synth.shard_kv_heads(synth.make_workload(spec, device, **kw), rank, world)
+    return synth.make_workload(rank_spec(spec, rank, world), device, **kw)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(script: str, argv, world: int, timeout_s: float = 3600.0) -> int:
+    """Starts `world` processes of `python script argv...`, one per rank, with RANK / LOCAL_RANK /
+    WORLD_SIZE / MASTER_ADDR / MASTER_PORT set, and waits for them.  Returns 0 only if every rank
+    exited 0; as soon as one fails (or the time runs out) the others are terminated, so that a job with
+    fewer ranks than asked for never reports a result."""
+    port = free_port()
+    procs = []
+    for r in range(world):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(world),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "INFO")               # the communicator's own log shows the rank count
+        env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        procs.append(subprocess.Popen([sys.executable, script, *argv], env=env))
+    deadline = time.time() + timeout_s
+    rc = 0
+    while procs and rc == 0:
+        for pr in list(procs):
+            code = pr.poll()
+            if code is not None:
+                procs.remove(pr)
+                if code != 0:
+                    rc = code if code > 0 else 1
+        if time.time() > deadline:
+            rc = 124
+        time.sleep(0.05)
+    for pr in procs:                                       # only after a failure: stop exactly what we started
+        pr.terminate()
+    for pr in procs:
+        try:
+            pr.wait(timeout=10)
+        except subprocess.TimeoutExpired:
+            pr.kill()
+    return rc
+
+
+def init_ranks(gpus: int, backend: str | None = None):
+    """Reads this process's place in the job from the environment, joins the process group when there
+    is more than one rank and returns (rank, local_rank, world, device).  The world size must be the
+    --gpus the run was asked for.  backend None: nccl on cuda:LOCAL_RANK; "gloo": CPU (host-side tests)."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != gpus:
+        raise SystemExit(f"bench.py: --gpus {gpus} but the job has {world} rank(s)")
+    if backend == "gloo":
+        dev = torch.device("cpu")
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+        if local >= torch.cuda.device_count():
+            raise SystemExit(f"bench.py: rank {rank} has no GPU (LOCAL_RANK {local}, {torch.cuda.device_count()} visible)")
+        torch.cuda.set_device(local)
+        dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if backend == "gloo":
+            dist.init_process_group("gloo", rank=rank, world_size=world)
+        else:
+            dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+        if dist.get_world_size() != gpus:
+            raise SystemExit(f"bench.py: process group has {dist.get_world_size()} ranks, {gpus} asked for")
+    return rank, local, world, dev
+
+
 def over_ranks(values, op, device):
     """Element-wise MAX or SUM of a list of floats over all ranks (identity without a process group)."""
     import torch
@@ -330,16 +426,7 @@ def run_cascade(args):
     import synth
     import paper_2510_07356_b200 as P
 
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    rank, local, world, dev = init_ranks(args.gpus)
     cw = synth.make_named_cascade(args.workload, dev)
     w, spec = cw.w, cw.w.spec
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
@@ -459,16 +546,7 @@ def run_prefill(args):
     import synth
     import paper_2510_07356_b200 as P
 
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    rank, local, world, dev = init_ranks(args.gpus)
     pw = synth.make_named_prefill(args.workload, dev)
     w, spec = pw.w, pw.w.spec
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
@@ -640,9 +718,16 @@ def run_curate(args):
 
 def main():
     args = parse_args()
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
     if args.impl == "reference":
         run_reference(args)
         return
+    if args.shard == "kv-heads" and args.workload.startswith(("casc", "prefill", "curate")):
+        raise SystemExit("bench.py: --shard kv-heads is implemented for the plain decode workloads")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no outside launcher: this process becomes the launcher of its own N ranks
+        raise SystemExit(spawn_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     if args.workload.startswith("casc"):
         run_cascade(args)
         return
@@ -657,23 +742,17 @@ def main():
     import torch.distributed as dist
     import synth
     import paper_2510_07356_b200 as P
+    from paper_2510_07356_b200 import bench_probe
 
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    rank, local, world, dev = init_ranks(args.gpus)
 
-    # every rank decodes its own batch of the same shape (replicas, no data-path collective)
-    spec = rank_spec(synth.SPECS[args.workload], rank, world)
-    w = synth.make_workload(spec, dev, spare_tokens=args.loop_steps)
+    # replicas: every rank decodes its own batch of the same shape; kv-heads: the ranks split one batch
+    # over its KV heads.  Neither has a data-path collective.
+    w = rank_workload(synth.SPECS[args.workload], rank, world, args.shard, dev, spare_tokens=args.loop_steps)
+    spec = w.spec
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local,
-                             num_q_heads=spec.num_q_heads, kv_layout=args.kv_layout)
+                             num_q_heads=spec.num_q_heads, num_kv_heads=spec.num_kv_heads,
+                             kv_layout=args.kv_layout)
     if args.kv_layout == 1:              # the same cache as [page][slot][KV head][D]
         w.k_pages = w.k_pages.permute(0, 2, 1, 3).contiguous()
         w.v_pages = w.v_pages.permute(0, 2, 1, 3).contiguous()
@@ -827,8 +906,8 @@ def main():
         chk_s = torch.zeros(2, dtype=torch.int32, device=dev)
 
         def probe_s():
-            P.concur_hbm_read_probe(w.k_pages, w.k_pages.numel() * 2, chk_s[0:1], 0, stream.cuda_stream)
-            P.concur_hbm_read_probe(w.v_pages, w.v_pages.numel() * 2, chk_s[1:2], 0, stream.cuda_stream)
+            bench_probe.read_probe(w.k_pages, w.k_pages.numel() * 2, chk_s[0:1], 0, stream.cuda_stream)
+            bench_probe.read_probe(w.v_pages, w.v_pages.numel() * 2, chk_s[1:2], 0, stream.cuda_stream)
 
         probe_ms, _, _ = back_to_back(probe_s, ms_per_step, args.sustained_seconds / 2)
         sustained["read_stream_gbs"] = pool_b / (probe_ms * 1e-3) / 1e9
@@ -840,8 +919,8 @@ def main():
         chk = torch.zeros(2, dtype=torch.int32, device=dev)
 
         def probe():
-            P.concur_hbm_read_probe(w.k_pages, w.k_pages.numel() * 2, chk[0:1], 0, stream.cuda_stream)
-            P.concur_hbm_read_probe(w.v_pages, w.v_pages.numel() * 2, chk[1:2], 0, stream.cuda_stream)
+            bench_probe.read_probe(w.k_pages, w.k_pages.numel() * 2, chk[0:1], 0, stream.cuda_stream)
+            bench_probe.read_probe(w.v_pages, w.v_pages.numel() * 2, chk[1:2], 0, stream.cuda_stream)
 
         for _ in range(3):
             probe()
@@ -853,7 +932,7 @@ def main():
         barrier()
         probe_ms = over_ranks([e0.elapsed_time(e1) / 10], "max", dev)[0]
         read_stream = {"gbs": pool_bytes / (probe_ms * 1e-3) / 1e9, "bytes": pool_bytes, "ms": probe_ms,
-                       "what": "concur_hbm_read_probe over k_pages then v_pages (16-byte loads, xor checksum), 10 passes"}
+                       "what": "read-only stream kernel of the bench's helper library over k_pages then v_pages (16-byte loads, xor checksum), 10 passes"}
 
     # ---- decode loop: KV append + attention per step, replayed from one CUDA graph
     loop = None
@@ -896,15 +975,18 @@ def main():
         traffic = MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN * w.kv_tokens     # scaled from the quarter-size capture
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": spec.name, "seed": spec.seed, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
+        "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if (args.shard == "kv-heads" and world > 1) else "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "warmup_requested": args.warmup,
+        "config": {"workload": args.workload, "rank0_shard": spec.name, "seed": spec.seed, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
                    "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128, "algorithmic_bytes": nbytes,
                    "l2": "flushed between steps (256 MB written, then 256 MB read)" if flush_needed else "inputs larger than L2",
                    "kernel": "mma" if args.kernel == 0 else "scalar", "ranges": R, "tiles": W,
                    "kv_layout": "token-major" if args.kv_layout == 1 else "head-major",
-                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
-        "kv_tokens_per_s": job_tokens / (ms_per_step * 1e-3),
+                   "parallelism": "1 gpu" if world == 1 else
+                                  (f"kv-heads x{world} ({spec.num_kv_heads} KV heads per rank)" if args.shard == "kv-heads"
+                                   else f"replicas x{world}")},
+        "kv_tokens_per_s": (w.kv_tokens if args.shard == "kv-heads" else job_tokens) / (ms_per_step * 1e-3),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -317,17 +317,6 @@ int concur_decode_attn_static(const void* q, const void* k_pages, const void* v_
                               int32_t batch, int32_t num_pages, int32_t block_table_stride,
                               int32_t page_size, void* cuda_stream);
 
-/* Measurement aid, not a step of the method (the paper has no counterpart): a read-only stream
- * over a device buffer.  Reads `bytes` bytes at `buf` (device, 16-byte aligned, `bytes` a
- * multiple of 16) exactly once with 16-byte loads and leaves the xor of all their 32-bit
- * words in `*checksum` (device, 4-byte aligned; zeroed by the call first).  A decode step is a
- * read-only scan of the KV cache, so this kernel's rate over the same pools is the plain-
- * stream figure to hold the partial kernel against (a device copy also writes).  `ctas` = grid
- * size, 0 = four CTAs of 512 threads per SM of the current device.  Asynchronous on
- * `cuda_stream`; allocates nothing.  Misaligned or null arguments are CONCUR_ERR_INVALID_ARG.
- */
-int concur_hbm_read_probe(const void* buf, size_t bytes, uint32_t* checksum, int32_t ctas, void* cuda_stream);
-
 /* Frees the handle and any memory the library allocated for it.  NULL is accepted. */
 int concur_attn_destroy(concur_attn_t* handle);
 

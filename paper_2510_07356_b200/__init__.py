@@ -10,7 +10,7 @@ attribute access without the library raises ImportError: there is no fallback.
 """
 import importlib
 
-_LAZY_MODULES = ("binding", "runner", "build")
+_LAZY_MODULES = ("binding", "runner", "build", "bench_probe")
 
 
 def _load_all():

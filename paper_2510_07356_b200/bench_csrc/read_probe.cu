@@ -3,10 +3,13 @@
 // cache, so the rate of this kernel over the same pools is the closest plain-stream yardstick for
 // the partial kernel (a device-to-device copy, the usual yardstick, also writes what it reads).
 // The checksum makes the reads observable, and lets a test check that every word was read once.
+//
+// Built into its own shared library (libconcur_bench.so) for the benchmark: it is no step of the
+// attention path and no part of the attention library's ABI.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "../../include/concur_attn.h"
+#include "read_probe.h"
 
 namespace concur {
 
@@ -47,28 +50,28 @@ __global__ void __launch_bounds__(kProbeThreads) read_probe_kernel(const uint4* 
 
 }  // namespace concur
 
-extern "C" int concur_hbm_read_probe(const void* buf, size_t bytes, uint32_t* checksum, int32_t ctas,
-                                     void* cuda_stream) {
-    if (!buf || !checksum || ctas < 0 || ctas > 65536) return CONCUR_ERR_INVALID_ARG;
+extern "C" int concur_bench_read_probe(const void* buf, size_t bytes, uint32_t* checksum, int32_t ctas,
+                                       void* cuda_stream) {
+    if (!buf || !checksum || ctas < 0 || ctas > 65536) return CONCUR_BENCH_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(buf) & 15u) || (bytes & 15u) || (reinterpret_cast<uintptr_t>(checksum) & 3u))
-        return CONCUR_ERR_INVALID_ARG;
+        return CONCUR_BENCH_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (ctas == 0) {
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
             cudaGetLastError();
-            return CONCUR_ERR_CUDA;
+            return CONCUR_BENCH_ERR_CUDA;
         }
         ctas = sms * 4;                       // four resident CTAs of 512 threads fill an SM's 2,048 thread slots
     }
     if (cudaMemsetAsync(checksum, 0, sizeof(uint32_t), stream) != cudaSuccess) {
         cudaGetLastError();
-        return CONCUR_ERR_CUDA;
+        return CONCUR_BENCH_ERR_CUDA;
     }
-    if (bytes == 0) return CONCUR_OK;
+    if (bytes == 0) return CONCUR_BENCH_OK;
     concur::read_probe_kernel<<<ctas, concur::kProbeThreads, 0, stream>>>(static_cast<const uint4*>(buf), bytes / 16,
                                                                           checksum);
-    if (cudaGetLastError() != cudaSuccess) return CONCUR_ERR_CUDA;
-    return CONCUR_OK;
+    if (cudaGetLastError() != cudaSuccess) return CONCUR_BENCH_ERR_CUDA;
+    return CONCUR_BENCH_OK;
 }

@@ -43,7 +43,7 @@ EXPORTS = (
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
     "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade", "concur_prefill_attn",
-    "concur_curate", "concur_hbm_read_probe",
+    "concur_curate",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -103,8 +103,6 @@ def _load() -> ctypes.CDLL:
     lib.concur_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_kv_append.restype = ctypes.c_int
     lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
-    lib.concur_hbm_read_probe.restype = ctypes.c_int
-    lib.concur_hbm_read_probe.argtypes = [vp, ctypes.c_size_t, vp, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
     lib.concur_attn_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.concur_attn_set_option.restype = ctypes.c_int
@@ -233,14 +231,6 @@ def concur_curate(params: concur_curate_params_t, correct, t_torch, t_kernel, le
                            _addr(pick), _addr(keep), _addr(difficulty), _addr(stats), stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_curate")
-    return rc
-
-
-def concur_hbm_read_probe(buf, nbytes, checksum, ctas=0, stream=0, check=True) -> int:
-    """Read-only stream over `nbytes` bytes of the device tensor `buf`; xor of its 32-bit words -> checksum[0]."""
-    rc = lib.concur_hbm_read_probe(_addr(buf), int(nbytes), _addr(checksum), int(ctas), stream or None)
-    if check and rc != CONCUR_OK:
-        raise ConcurError(rc, "concur_hbm_read_probe")
     return rc
 
 

@@ -61,6 +61,13 @@ SPECS = {
     # config 3 with 40 query heads (group size 5): the geometry variant of the same workload
     "cfg3h40_b64_ctx16384_p64": Spec("cfg3h40_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563,
                                      num_q_heads=40),
+    # what one rank of config 3 holds when the model is tensor-parallel over its KV heads on 8 / 4 / 2 GPUs
+    "cfg3kv1_b64_ctx16384_p64": Spec("cfg3kv1_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563,
+                                     num_q_heads=8, num_kv_heads=1),
+    "cfg3kv2_b64_ctx16384_p64": Spec("cfg3kv2_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563,
+                                     num_q_heads=16, num_kv_heads=2),
+    "cfg3kv4_b64_ctx16384_p64": Spec("cfg3kv4_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563,
+                                     num_q_heads=32, num_kv_heads=4),
     "cfg4_b256_logu2k_32k_p64": Spec("cfg4_b256_logu2k_32k_p64", 256, 64, ("loguniform", 2048, 32768), seed=73564),
     "cfg5_b32_skew128k_p64": Spec("cfg5_b32_skew128k_p64", 32, 64, ("skew", 131072, 256, 4096),
                                   k_outlier_prob=0.01, seed=73565),

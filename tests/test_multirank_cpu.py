@@ -1,53 +1,84 @@
-"""The N > 1 path of the benchmark on CPU: two gloo ranks run the replica sharding and the
-max / sum over ranks that bench.py uses (the data path itself has no collective)."""
+"""The N > 1 path of the benchmark on CPU: bench.py's own launcher starts two gloo ranks, which take
+their shares through bench.rank_workload and reduce through bench.over_ranks (the data path itself has
+no collective; with no GPU here each rank's share is computed by the CPU oracle)."""
 import os
-import socket
+import subprocess
 import sys
 
 import numpy as np
-import torch
-import torch.distributed as dist
-import torch.multiprocessing as mp
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+WORKER = os.path.join(ROOT, "tests", "bench_rank_worker.py")
+sys.path.insert(0, ROOT)
 
 
-def _free_port():
-    with socket.socket() as s:
-        s.bind(("127.0.0.1", 0))
-        return s.getsockname()[1]
+def _load(tmp_path, world):
+    return [np.load(tmp_path / f"rank{r}.npz") for r in range(world)]
 
 
-def _worker(rank, world, port, out_dir):
-    sys.path.insert(0, ROOT)
-    os.environ["MASTER_ADDR"] = "127.0.0.1"
-    os.environ["MASTER_PORT"] = str(port)
-    dist.init_process_group("gloo", rank=rank, world_size=world)
+def test_kv_head_shards_of_two_ranks_put_together_equal_the_unsharded_oracle(tmp_path):
     import bench
+    import oracle
     import synth
-    spec = bench.rank_spec(synth.SPECS["cfg2_b16_u1k_8k_p16"], rank, world)
-    lens = synth.make_lengths(spec)
-    ms = 1.0 + rank                                   # rank 1 is the slow one
-    mx = bench.over_ranks([ms, 10.0 - rank], "max", "cpu")
-    sm = bench.over_ranks([float(lens.sum()), 1.0], "sum", "cpu")
-    np.save(os.path.join(out_dir, f"r{rank}.npy"), np.array([spec.seed, lens.sum(), *mx, *sm], dtype=np.float64))
-    dist.barrier()
-    dist.destroy_process_group()
-
-
-def test_two_gloo_ranks_shard_and_reduce(tmp_path):
     world = 2
-    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
-    r0 = np.load(tmp_path / "r0.npy")
-    r1 = np.load(tmp_path / "r1.npy")
-    assert r0[0] != r1[0] and r0[1] != r1[1]           # replicas draw different batches
-    for r in (r0, r1):
-        assert r[2] == 2.0 and r[3] == 10.0            # max over ranks (time of the slowest rank)
-        assert r[4] == r0[1] + r1[1] and r[5] == 2.0   # units all ranks processed
+    rc = bench.spawn_ranks(WORKER, ["--gpus", str(world), "--shard", "kv-heads", "--out", str(tmp_path)], world,
+                           timeout_s=300)
+    assert rc == 0
+    r = _load(tmp_path, world)
+    full = synth.make_workload(synth.tiny_spec("ranks", (300, 1, 0, 64, 777, 1300), 16, 9100), "cpu")
+    ref_out, ref_lse = oracle.decode_attn(full.q, full.k_pages, full.v_pages, full.block_table, full.seq_lens,
+                                          full.scale)
+    assert [int(x["hkv"]) for x in r] == [4, 4] and [int(x["hq"]) for x in r] == [32, 32]
+    # query heads 0..31 belong to rank 0 (KV heads 0..3), 32..63 to rank 1: side by side they are the
+    # whole result, bit for bit (a head's result depends on nothing outside its own KV head)
+    assert np.array_equal(np.concatenate([x["out"] for x in r], axis=1), ref_out, equal_nan=True)
+    assert np.array_equal(np.concatenate([x["lse"] for x in r], axis=1), ref_lse)
+    for x in r:
+        assert x["max_ms"] == 2.0 and int(x["world"]) == 2              # time of the slowest rank
+        assert x["sum_bytes"] == float(r[0]["bytes"]) + float(r[1]["bytes"])
+    # K and V bytes are split, tables and lengths are read by both
+    assert r[0]["sum_bytes"] > full.algorithmic_bytes() - 1 and r[0]["sum_bytes"] < full.algorithmic_bytes() + 4096
+
+
+def test_replica_ranks_draw_their_own_batches(tmp_path):
+    import bench
+    world = 2
+    rc = bench.spawn_ranks(WORKER, ["--gpus", str(world), "--shard", "replicas", "--out", str(tmp_path)], world,
+                           timeout_s=300)
+    assert rc == 0
+    r = _load(tmp_path, world)
+    assert int(r[0]["seed"]) != int(r[1]["seed"]) and int(r[0]["hkv"]) == 8
+    assert not np.array_equal(r[0]["out"], r[1]["out"], equal_nan=True)
+    assert r[0]["sum_tokens"] == r[1]["sum_tokens"] == 2 * (300 + 1 + 64 + 777 + 1300)
+
+
+def test_a_failing_rank_fails_the_job(tmp_path):
+    import bench
+    rc = bench.spawn_ranks(WORKER, ["--gpus", "2", "--out", str(tmp_path), "--fail-rank", "1"], 2, timeout_s=300)
+    assert rc != 0
+
+
+def test_world_size_must_match_gpus(tmp_path):
+    import bench
+    # two ranks started, three asked for: every rank refuses
+    rc = bench.spawn_ranks(WORKER, ["--gpus", "3", "--out", str(tmp_path)], 2, timeout_s=300)
+    assert rc != 0
+    assert not list(tmp_path.glob("rank*.npz"))
+
+
+def test_bench_cli_launches_its_own_ranks_and_fails_without_gpus():
+    import torch
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        return                                   # on a multi-GPU machine this would be a real run
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE")}
+    pr = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1", "--warmup", "0",
+                         "--workload", "cfg1_b1_ctx512_p16", "--no-cpu", "--no-e2e"],
+                        env=env, capture_output=True, text=True, timeout=600)
+    assert pr.returncode != 0                    # fewer GPUs than ranks: no result line, non-zero exit
+    assert '"metric"' not in pr.stdout
 
 
 def test_single_process_reductions_are_identity():
-    sys.path.insert(0, ROOT)
     import bench
     import synth
     assert bench.over_ranks([3.0, 4.0], "max", "cpu") == [3.0, 4.0]
