@@ -530,6 +530,164 @@ def run_cascade(args):
         dist.destroy_process_group()
 
 
+def run_loop(args):
+    """A token step of a model with L layers, replayed from one CUDA graph: per layer the new token's
+    K/V rows are appended to that layer's pools and the layer's decode attention runs on them; the
+    lengths (one set for all layers) grow by one per replay.  `loop<L>_<decode workload>`."""
+    import torch
+    import synth
+    import paper_2510_07356_b200 as P
+
+    rank, local, world, dev = init_ranks(args.gpus)
+    head, base_name = args.workload.split("_", 1)
+    L = int(head[len("loop"):])
+    base = rank_spec(synth.SPECS[base_name], rank, world)
+    K, W_ = args.steps, max(3, args.warmup)
+    replays = 2 * (W_ + K) + 8                           # interleaved, attention-only, eager passes
+    ws = [synth.make_workload(base, dev, spare_tokens=replays, value_seed=base.seed + 7919 * i) for i in range(L)]
+    w0 = ws[0]
+    spec = w0.spec
+    B, stride = spec.batch, w0.block_table.shape[1]
+    attn = P.DecodeAttention(spec.page_size, B, stride, local, num_q_heads=spec.num_q_heads,
+                             num_kv_heads=spec.num_kv_heads)
+    g = torch.Generator(device=dev); g.manual_seed(base.seed + 17)
+    kn = torch.randn((L, B, spec.num_kv_heads, spec.head_dim), generator=g, device=dev).to(torch.bfloat16)
+    vn = torch.randn((L, B, spec.num_kv_heads, spec.head_dim), generator=g, device=dev).to(torch.bfloat16)
+    lens = w0.seq_lens.clone()
+    outs = [torch.empty_like(w0.q) for _ in range(L)]
+    lses = [torch.empty((B, spec.num_q_heads), dtype=torch.float32, device=dev) for _ in range(L)]
+    stream = torch.cuda.current_stream(dev)
+    flush = L2Flush(dev)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def append(i, s_):
+        P.concur_kv_append_layer(attn.handle, kn[i], vn[i], ws[i].k_pages, ws[i].v_pages, w0.block_table, lens, B,
+                                 w0.num_pages, stride, 1 if i == 0 else 0, s_)
+
+    def attend(i, s_):
+        P.concur_decode_attn(attn.handle, ws[i].q, ws[i].k_pages, ws[i].v_pages, w0.block_table, lens, w0.scale,
+                             outs[i], lses[i], B, w0.num_pages, stride, s_)
+
+    def token_step():                                    # what a model does: layer by layer
+        s_ = torch.cuda.current_stream(dev).cuda_stream
+        for i in range(L):
+            append(i, s_)
+            attend(i, s_)
+
+    def attention_chain():                               # the L attention calls alone, back to back
+        s_ = torch.cuda.current_stream(dev).cuda_stream
+        for i in range(L):
+            attend(i, s_)
+
+    def capture(fn):
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            fn()                                         # first-call set-up stays outside the capture
+        stream.wait_stream(side)
+        torch.cuda.synchronize(dev)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fn()
+        return graph
+
+    def timed(graph, n):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n)]
+        for row in ev:
+            for e in row:
+                e.record(stream)
+        barrier()
+        for i in range(n):
+            flush()                                      # every replay starts with none of the pools in L2
+            ev[i][0].record(stream)
+            graph.replay()
+            ev[i][1].record(stream)
+        barrier()
+        return [ev[i][0].elapsed_time(ev[i][1]) for i in range(n)]
+
+    results = {}
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    clocks = None
+    for name, fn, overlap in (("interleaved", token_step, 0), ("attention_only", attention_chain, 0),
+                              ("attention_only_overlapped", attention_chain, 1)):
+        attn.set_option(P.CONCUR_OPT_OVERLAP_CALLS, overlap)
+        graph = capture(fn)
+        timed(graph, W_)
+        if name == "interleaved" and rank == 0:
+            sampler.start(); time.sleep(0.2)
+        t0m = time.time()
+        ms = timed(graph, K)
+        if name == "interleaved" and rank == 0:
+            clocks = sampler.stop(t0m, time.time())
+        results[name] = over_ranks([sum(ms) / K, min(ms)], "max", dev)
+        del graph
+    attn.set_option(P.CONCUR_OPT_OVERLAP_CALLS, 0)
+    assert attn.status() == 0, "device-side flags set"
+    # the partial kernel alone, eagerly, with the library's events around it (one pass over the layers)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(L)]
+    for row in ev:
+        for e in row:
+            e.record(stream)
+    part = []
+    for _ in range(2):
+        flush()
+        for i in range(L):
+            attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, ev[i][0].cuda_event)
+            attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, ev[i][1].cuda_event)
+            attend(i, stream.cuda_stream)
+        barrier()
+        part = [ev[i][0].elapsed_time(ev[i][1]) for i in range(L)]
+    attn.set_option(P.CONCUR_OPT_EVENT_BEFORE_PARTIAL, 0)
+    attn.set_option(P.CONCUR_OPT_EVENT_AFTER_PARTIAL, 0)
+    part_ms = over_ranks([sum(part) / L], "max", dev)[0]
+    # parity of the last layer, as the loop left it, against the oracle (one-GPU runs)
+    lens_now = lens.cpu().numpy().astype("int32")
+    w_last = ws[L - 1]
+    w_last.seq_lens = lens.clone(); w_last.lens_host = lens_now
+    token_bytes = 2 * spec.num_kv_heads * spec.head_dim * 2
+    layer_bytes = w_last.algorithmic_bytes() + B * token_bytes       # the layer's attention plus its appended rows
+    job_bytes = over_ranks([float(layer_bytes) * L], "sum", dev)[0]
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    peak, peak_kind = measured_peak()
+    ms_step, ms_min = results["interleaved"]
+    achieved = w_last.algorithmic_bytes() / (part_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": job_bytes / (ms_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W_, "warmup_requested": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "layers": L, "batch": B, "kv_tokens_per_layer": int(lens_now.sum()),
+                   "page_size": spec.page_size, "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128,
+                   "algorithmic_bytes_per_layer": layer_bytes,
+                   "l2": "flushed before every replay (256 MB written, then 256 MB read)",
+                   "step": "one CUDA graph: per layer concur_kv_append_layer + concur_decode_attn (one launch each)",
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+        "us_per_layer": ms_step * 1e3 / L, "us_per_layer_min": ms_min * 1e3 / L,
+        "attention_only_us_per_layer": results["attention_only"][0] * 1e3 / L,
+        "attention_only_overlapped_us_per_layer": results["attention_only_overlapped"][0] * 1e3 / L,
+        "frac_of_measured_copy": job_bytes / world / (ms_step * 1e-3) / 1e9 / peak,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "partial (mean over the layers, eager pass)",
+                     "ms": part_ms},
+        "e2e": None, "gpu_launches": 2 * L * K, "clocks": clocks,
+    }
+    if not args.no_cpu and world == 1:
+        line["cpu_baseline"], line["parity"] = cpu_baseline(w_last, args.cpu_seconds, (outs[L - 1], lses[L - 1]))
+    print(json.dumps(line), flush=True)
+
+
 def measured_tensor_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -723,11 +881,14 @@ def main():
     if args.impl == "reference":
         run_reference(args)
         return
-    if args.shard == "kv-heads" and args.workload.startswith(("casc", "prefill", "curate")):
+    if args.shard == "kv-heads" and args.workload.startswith(("casc", "prefill", "curate", "loop")):
         raise SystemExit("bench.py: --shard kv-heads is implemented for the plain decode workloads")
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # no outside launcher: this process becomes the launcher of its own N ranks
         raise SystemExit(spawn_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
+    if args.workload.startswith("loop"):
+        run_loop(args)
+        return
     if args.workload.startswith("casc"):
         run_cascade(args)
         return
@@ -959,7 +1120,8 @@ def main():
         barrier()
         loop_ms = over_ranks([e0.elapsed_time(e1) / args.loop_steps], "max", dev)[0]
         assert int(lens_loop[0]) == int(w.lens_host[0]) + args.loop_steps
-        loop = {"steps": args.loop_steps, "ms_per_step": loop_ms, "launches_per_step": 3,
+        loop = {"steps": args.loop_steps, "ms_per_step": loop_ms,
+                "launches_per_step": 2 if (args.kernel == 0 and args.fuse_combine != 0 and spec.batch <= 511) else 3,
                 "what": "concur_kv_append + concur_decode_attn replayed from a CUDA graph, lengths +1 per step"}
 
     if rank != 0:
@@ -970,6 +1132,10 @@ def main():
     peak, peak_kind = measured_peak()
     value = job_bytes / (ms_per_step * 1e-3) / 1e9
     achieved = nbytes / (part_ms_avg * 1e-3) / 1e9
+    # the tensor-core kernel with the merge fused is the whole step for up to 511 sequences; beyond that a
+    # plan kernel runs ahead of it; the scalar kernel, or an unfused merge, adds the combine kernel
+    fused = args.kernel == 0 and args.fuse_combine != 0
+    launches_per_step = (1 if spec.batch <= 511 else 2) if fused else 3
     traffic = None
     if args.kernel == 0 and spec.page_size == 64 and MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN:
         traffic = MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN * w.kv_tokens     # scaled from the quarter-size capture
@@ -996,7 +1162,7 @@ def main():
         "sustained": sustained,
         "read_stream": read_stream,
         "frac_of_measured_read_stream": (achieved / read_stream["gbs"]) if read_stream else None,
-        "decode_loop": loop, "e2e": e2e, "gpu_launches": (2 if args.kernel == 0 else 3) * K, "clocks": clocks, "device_flags": flags,
+        "decode_loop": loop, "e2e": e2e, "gpu_launches": launches_per_step * K, "clocks": clocks, "device_flags": flags,
     }
     if not args.no_cpu and world == 1:       # the oracle leg belongs to the one-GPU run
         step()                                   # the inputs as they are now, once more, for the comparison

@@ -61,7 +61,9 @@ typedef enum {
 /* Sticky device-side condition bits reported by concur_attn_status. */
 #define CONCUR_FLAG_BAD_PAGE_ID 1u  /* a used block-table entry was outside [0, num_pages): clamped    */
 #define CONCUR_FLAG_BAD_SEQ_LEN 2u  /* a seq_lens entry was outside [0, stride*P]: clamped             */
-#define CONCUR_FLAG_WAIT_LIMIT  4u  /* an in-kernel wait gave up; results of that call are invalid      */
+#define CONCUR_FLAG_WAIT_LIMIT  4u  /* an in-kernel wait gave up; results of that call are invalid, and so
+                                       are those of later calls on the handle until concur_attn_status
+                                       has reported the flag (it then re-initialises the handle's counters) */
 #define CONCUR_FLAG_BAD_GROUP   8u  /* cascade step: group_start was not 0 <= g[0] <= g[1] <= ... <= batch;
                                        the call then shared nothing and computed the plain step          */
 
@@ -89,6 +91,24 @@ typedef enum {
 #define CONCUR_OPT_SMALL_PAGE_COPY 11 /* tensor-core partial kernel with 16- or 32-token pages: 1 (default) = the
                                         producer warp copies tiles 16 bytes per lane, 0 = one TMA box per
                                         (page, head) chunk                                               */
+
+#define CONCUR_OPT_WAIT_LIMIT_NS 12 /* tensor-core partial kernel: nanoseconds after which a warp's wait for
+                                       another role of its CTA (a tile to land, a ring stage to be freed, a
+                                       partial to merge) gives up.  The kernel then records
+                                       CONCUR_FLAG_WAIT_LIMIT, every warp of that CTA returns once the copies it
+                                       has in flight have landed, and the call's results are invalid; nothing
+                                       faults and the handle stays usable.  0 = default (2 s; 60 s at most).
+                                       No correct run comes near the default; the option exists so that the
+                                       give-up path can be exercised                                       */
+
+#define CONCUR_OPT_OVERLAP_CALLS 13 /* 1 = a decode call that is a single kernel launch (see concur_decode_attn) may
+                                       start while the kernel ahead of it on the stream drains, if that kernel
+                                       is such a call too: its CTAs take over the SMs the earlier call's CTAs
+                                       leave and fill their rings, and write nothing before the earlier call
+                                       has finished.  The caller promises that q, the pools, block_table and
+                                       seq_lens of a call are not written by the call right ahead of it (true
+                                       of the layers of a model, whose calls differ in q, pools and out).
+                                       0 (default) = calls run strictly one after the other              */
 
 /* Layouts of the K and V pools (concur_attn_config_t.kv_layout). */
 #define CONCUR_KV_HEAD_MAJOR  0   /* [num_pages][Hkv][P][D]: one (page, head) tile is contiguous (default) */
@@ -140,6 +160,11 @@ int concur_attn_create(const concur_attn_config_t* cfg, concur_attn_t** handle);
  *   num_pages                  pages in each pool, >= 1
  *   block_table_stride         int32 elements per table row, 1 .. max_pages_per_seq
  *
+ * Launches: one kernel for batches of up to 511 sequences (the partial kernel works the plan out for
+ * itself from seq_lens, merges split sequences itself and leaves the workspace ready for the next
+ * call); a plan kernel and the partial kernel beyond that, unless the plan was made ahead with
+ * concur_attn_plan; a third (combine) kernel only with the scalar kernel or CONCUR_OPT_FUSE_COMBINE 0.
+ *
  * Errors: CONCUR_ERR_INVALID_ARG (null or misaligned pointer, bad size),
  * CONCUR_ERR_TOO_LARGE (batch or stride above the handle's limits), CONCUR_ERR_CUDA
  * (launch failure).  Bad *contents* never fault: a page id outside [0, num_pages) or a
@@ -152,6 +177,34 @@ int concur_decode_attn(concur_attn_t* handle,
                        float scale, void* out, float* lse,
                        int32_t batch, int32_t num_pages, int32_t block_table_stride,
                        void* cuda_stream);
+
+/*
+ * Plan once per token step, attend once per layer.  All layers of a model see the same seq_lens in a
+ * decode step, so the split-KV plan (tile counts, ranges) is the same for each of them.  (The paper's
+ * generation runs, Sec. 3.3 and 4.2, are such loops over the layers of 32B models; the paper does not
+ * describe them.)
+ *
+ *   concur_attn_plan             computes the plan of (seq_lens, batch, block_table_stride) into the
+ *                                handle's workspace: one small kernel on `cuda_stream`.
+ *   concur_decode_attn_planned   concur_decode_attn as ONE kernel launch, using that plan.  It must
+ *                                follow, on the same stream, a concur_attn_plan call with the same
+ *                                seq_lens pointer, batch and stride, with no other call on the handle
+ *                                in between except further concur_decode_attn_planned and concur_kv_append
+ *                                calls; seq_lens' contents must be what the plan call saw (so: append all
+ *                                layers' rows with lengths advanced once, or plan after the append).
+ *                                Otherwise CONCUR_ERR_INVALID_ARG.  Batches of up to 511 sequences need
+ *                                no plan call at all (concur_decode_attn is already one launch there)
+ *                                and are accepted without one.
+ * Arguments, asynchrony and other errors as for concur_decode_attn.
+ */
+int concur_attn_plan(concur_attn_t* handle, const int32_t* seq_lens, int32_t batch,
+                     int32_t block_table_stride, void* cuda_stream);
+int concur_decode_attn_planned(concur_attn_t* handle,
+                               const void* q, const void* k_pages, const void* v_pages,
+                               const int32_t* block_table, const int32_t* seq_lens,
+                               float scale, void* out, float* lse,
+                               int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                               void* cuda_stream);
 
 /*
  * The same step when sequences share a cached prefix (cascade decode).  In the paper's
@@ -244,6 +297,20 @@ int concur_kv_append(concur_attn_t* handle, const void* k_new, const void* v_new
                      void* cuda_stream);
 
 /*
+ * The same write for the further layers of a model.  A model keeps one pair of pools per layer and one
+ * set of lengths for all of them, so only the step's first append may advance the lengths:
+ *   advance = 1   exactly concur_kv_append: rows go to position seq_lens[b], which becomes seq_lens[b] + 1;
+ *   advance = 0   rows go to position seq_lens[b] - 1 -- the slot the step's first append opened -- and
+ *                 seq_lens is only read.  A length of 0 (no slot opened) is flagged like any position
+ *                 outside the table row and nothing is written.
+ * Any other `advance` is CONCUR_ERR_INVALID_ARG; everything else as for concur_kv_append.
+ */
+int concur_kv_append_layer(concur_attn_t* handle, const void* k_new, const void* v_new,
+                           void* k_pages, void* v_pages, const int32_t* block_table, int32_t* seq_lens,
+                           int32_t batch, int32_t num_pages, int32_t block_table_stride, int32_t advance,
+                           void* cuda_stream);
+
+/*
  * The same step for callers whose tensors live in HOST memory (pinned memory gives
  * asynchronous copies).  Every pointer is a host pointer with the layouts above; the
  * library copies the inputs into device staging buffers that it owns (allocated on first
@@ -261,7 +328,8 @@ int concur_decode_attn_host(concur_attn_t* handle,
 /*
  * Synchronises `cuda_stream` and returns, in *flags (host pointer), the OR of the
  * CONCUR_FLAG_* conditions seen by any call on this handle since the last status call;
- * the device word is then cleared.
+ * the device word is then cleared.  If CONCUR_FLAG_WAIT_LIMIT is among them the handle's workspace
+ * counters are re-initialised as well, so that the next call starts clean.
  */
 int concur_attn_status(concur_attn_t* handle, void* cuda_stream, uint32_t* flags);
 

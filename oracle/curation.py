@@ -74,10 +74,12 @@ def pearson(length, sp, correct):
     n = x.size
     if n < 2:
         return float("nan"), n
-    sx, sy = x.sum(), y.sum()
-    cov = (x * y).sum() - sx * sy / n
-    vx = (x * x).sum() - sx * sx / n
-    vy = (y * y).sum() - sy * sy / n
+    # the textbook definition, centred on the means:
+    #   r = sum (x - mx)(y - my) / sqrt( sum (x - mx)^2 * sum (y - my)^2 )
+    dx, dy = x - x.mean(), y - y.mean()
+    cov = (dx * dy).sum()
+    vx = (dx * dx).sum()
+    vy = (dy * dy).sum()
     if not vx * vy > 0:                                  # a constant column: the coefficient is undefined
         return float("nan"), n
     return float(cov / np.sqrt(vx * vy)), n

@@ -8,13 +8,15 @@ from __future__ import annotations
 import numpy as np
 
 
-def kv_append(k_pages, v_pages, block_table, seq_lens, k_new, v_new):
+def kv_append(k_pages, v_pages, block_table, seq_lens, k_new, v_new, advance=True):
     """In place: stores k_new[b], v_new[b] ([Hkv][D]) at position seq_lens[b] and advances
     seq_lens[b].  A sequence whose position does not fit its table row, or whose page id is
-    outside the pool, is left untouched."""
+    outside the pool, is left untouched.  advance=False is the write of a further layer of the
+    same step: the rows go to the slot the step's first append opened, position seq_lens[b] - 1,
+    and the lengths stay."""
     num_pages, hkv, P, _ = k_pages.shape
     for b in range(len(seq_lens)):
-        pos = int(seq_lens[b])
+        pos = int(seq_lens[b]) - (0 if advance else 1)
         if pos < 0 or pos >= block_table.shape[1] * P:
             continue
         page = int(block_table[b, pos // P])
@@ -23,7 +25,8 @@ def kv_append(k_pages, v_pages, block_table, seq_lens, k_new, v_new):
         for g in range(hkv):
             k_pages[page, g, pos % P, :] = k_new[b, g, :]
             v_pages[page, g, pos % P, :] = v_new[b, g, :]
-        seq_lens[b] = pos + 1
+        if advance:
+            seq_lens[b] = pos + 1
 
 
 def gather_tokens(pool, block_table, b, n):

@@ -37,13 +37,16 @@ CONCUR_OPT_FUSE_COMBINE = 8
 CONCUR_OPT_CLAIM_AHEAD = 9
 CONCUR_OPT_PREFIX_KERNEL = 10
 CONCUR_OPT_SMALL_PAGE_COPY = 11
+CONCUR_OPT_WAIT_LIMIT_NS = 12
+CONCUR_OPT_OVERLAP_CALLS = 13
 
 EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",
     "concur_decode_attn_host", "concur_attn_status", "concur_attn_set_option",
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
     "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade", "concur_prefill_attn",
-    "concur_curate",
+    "concur_curate", "concur_attn_plan", "concur_decode_attn_planned",
+    "concur_kv_append_layer",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -90,6 +93,10 @@ def _load() -> ctypes.CDLL:
     decode_args = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, vp]
     lib.concur_decode_attn.restype = ctypes.c_int
     lib.concur_decode_attn.argtypes = decode_args
+    lib.concur_decode_attn_planned.restype = ctypes.c_int
+    lib.concur_decode_attn_planned.argtypes = decode_args
+    lib.concur_attn_plan.restype = ctypes.c_int
+    lib.concur_attn_plan.argtypes = [vp, vp, i32, i32, vp]
     lib.concur_decode_attn_host.restype = ctypes.c_int
     lib.concur_decode_attn_host.argtypes = decode_args
     lib.concur_decode_attn_static.restype = ctypes.c_int
@@ -103,6 +110,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_kv_append.restype = ctypes.c_int
     lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
+    lib.concur_kv_append_layer.restype = ctypes.c_int
+    lib.concur_kv_append_layer.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
     lib.concur_attn_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.concur_attn_set_option.restype = ctypes.c_int
@@ -178,6 +187,22 @@ def concur_decode_attn(handle, q, k_pages, v_pages, block_table, seq_lens, scale
                    stream, check)
 
 
+def concur_attn_plan(handle, seq_lens, batch, block_table_stride, stream=0, check=True) -> int:
+    """The split-KV plan of one token step, for the concur_decode_attn_planned calls of its layers."""
+    rc = lib.concur_attn_plan(handle, _addr(seq_lens), batch, block_table_stride, stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_attn_plan")
+    return rc
+
+
+def concur_decode_attn_planned(handle, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
+                               batch, num_pages, block_table_stride, stream=0, check=True) -> int:
+    """concur_decode_attn as one launch, on the plan of the preceding concur_attn_plan call."""
+    return _decode(lib.concur_decode_attn_planned, "concur_decode_attn_planned", handle, q, k_pages, v_pages,
+                   block_table, seq_lens, scale, out, lse, batch, num_pages, block_table_stride,
+                   stream, check)
+
+
 def concur_decode_attn_host(handle, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
                             batch, num_pages, block_table_stride, stream=0, check=True) -> int:
     """Host tensors (pinned for asynchronous copies); synchronises before returning."""
@@ -242,6 +267,18 @@ def concur_kv_append(handle, k_new, v_new, k_pages, v_pages, block_table, seq_le
                               stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_kv_append")
+    return rc
+
+
+def concur_kv_append_layer(handle, k_new, v_new, k_pages, v_pages, block_table, seq_lens, batch, num_pages,
+                           block_table_stride, advance, stream=0, check=True) -> int:
+    """concur_kv_append for one layer of several: advance=1 for the step's first append, 0 for the others
+    (they write the slot the first one opened and leave seq_lens alone)."""
+    rc = lib.concur_kv_append_layer(handle, _addr(k_new), _addr(v_new), _addr(k_pages), _addr(v_pages),
+                                    _addr(block_table), _addr(seq_lens), batch, num_pages, block_table_stride,
+                                    int(advance), stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_kv_append_layer")
     return rc
 
 

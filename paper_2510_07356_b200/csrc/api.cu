@@ -5,6 +5,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "tensor_map.cuh"
 
 using namespace concur;
 
@@ -91,9 +92,15 @@ struct concur_attn {
     int32_t claim_ahead = 1 << 20;
     int32_t prefix_kernel = 0;
     int32_t small_page_copy = 1;
+    int64_t wait_limit_ns = 2000000000ll;
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;
     Staging st_q, st_k, st_v, st_bt, st_len, st_out, st_lse;
     Staging cascade_ws;          // allocated on the first cascade call
+    int32_t overlap_calls = 0;
+    RowsMapCache maps;           // tensor maps of the pools seen recently
+    // the plan concur_attn_plan left in the workspace, for concur_decode_attn_planned
+    const int32_t* planned_lens = nullptr;
+    int32_t planned_batch = -1, planned_stride = -1;
 };
 
 extern "C" {
@@ -129,8 +136,9 @@ int concur_attn_create(const concur_attn_config_t* cfg, concur_attn_t** handle) 
         h->ws = static_cast<char*>(p);
         h->owns_ws = true;
     }
-    // only the header must start defined; partial slots are written before they are read
-    if (cudaMemset(h->ws, 0, h->lay.prefix) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    // the header and the per-unit ticket counters must start at zero (a launch without a plan kernel relies
+    // on both); partial slots are written before they are read
+    if (cudaMemset(h->ws, 0, h->lay.part_lse) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
         if (h->owns_ws) cudaFree(h->ws);
         delete h; return CONCUR_ERR_CUDA;
     }
@@ -170,6 +178,8 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.max_ranges = kMaxRanges;
     p.fuse_combine = h->fuse_combine;
     p.claim_ahead = h->claim_ahead;
+    p.wait_limit_ns = h->wait_limit_ns;
+    p.overlap_next = h->overlap_calls;
     p.hdr = reinterpret_cast<int32_t*>(h->ws + h->lay.hdr);
     p.tiles_prefix = reinterpret_cast<int32_t*>(h->ws + h->lay.prefix);
     p.range_start = reinterpret_cast<int32_t*>(h->ws + h->lay.range_start);
@@ -197,10 +207,24 @@ static int check_call(concur_attn_t* h, const void* q, const void* k_pages, cons
     return CONCUR_OK;
 }
 
-static int enqueue(concur_attn_t* h, const DecodeParams& p, cudaStream_t stream) {
-    if (launch_plan(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+// The sequences whose plan the tensor-core partial kernel keeps in shared memory and can therefore work
+// out for itself (its kSmemBatch).
+constexpr int32_t kSelfPlanBatch = 511;
+
+// One launch instead of two: the tensor-core kernel with the merge fused needs no plan kernel when it
+// plans for itself (batch <= kSelfPlanBatch) or when the tables of a matching concur_attn_plan call are
+// in the workspace (`planned`).
+static bool single_launch(const concur_attn_t* h, int32_t batch, bool planned) {
+    return h->kernel == 0 && h->fuse_combine && (batch <= kSelfPlanBatch || planned);
+}
+
+static int enqueue(concur_attn_t* h, DecodeParams& p, cudaStream_t stream, bool planned = false) {
+    p.no_plan_launch = single_launch(h, p.batch, planned) ? 1 : 0;
+    // every launch but the one that reads them overwrites the tables a concur_attn_plan call left
+    if (!(planned && p.batch > kSelfPlanBatch)) h->planned_batch = -1;
+    if (!p.no_plan_launch && launch_plan(p, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if (h->ev_before && cudaEventRecord(h->ev_before, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
-    cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream);
+    cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream, &h->maps);
     if (e != cudaSuccess) return CONCUR_ERR_CUDA;
     if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     // the tensor-core kernel merges split units itself; the scalar kernel leaves that to the
@@ -224,10 +248,56 @@ int concur_decode_attn(concur_attn_t* h, const void* q, const void* k_pages, con
     return enqueue(h, p, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int concur_attn_plan(concur_attn_t* h, const int32_t* seq_lens, int32_t batch, int32_t block_table_stride,
+                     void* cuda_stream) {
+    if (!h) return CONCUR_ERR_INVALID_ARG;
+    if (batch < 0 || block_table_stride < 1) return CONCUR_ERR_INVALID_ARG;
+    if (batch > h->cfg.max_batch || block_table_stride > h->cfg.max_pages_per_seq) return CONCUR_ERR_TOO_LARGE;
+    h->planned_batch = -1;
+    if (batch == 0) return CONCUR_OK;
+    if (!seq_lens || !aligned(seq_lens, 4)) return CONCUR_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok()) return CONCUR_ERR_CUDA;
+    DecodeParams p = {};
+    fill_params(h, p, nullptr, nullptr, nullptr, nullptr, seq_lens, 1.f, nullptr, nullptr, batch, 1,
+                block_table_stride);
+    if (launch_plan(p, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return CONCUR_ERR_CUDA;
+    h->planned_lens = seq_lens;
+    h->planned_batch = batch;
+    h->planned_stride = block_table_stride;
+    return CONCUR_OK;
+}
+
+int concur_decode_attn_planned(concur_attn_t* h, const void* q, const void* k_pages, const void* v_pages,
+                               const int32_t* block_table, const int32_t* seq_lens, float scale, void* out,
+                               float* lse, int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                               void* cuda_stream) {
+    int rc = check_call(h, q, k_pages, v_pages, block_table, seq_lens, out, lse, batch, num_pages,
+                        block_table_stride, 16);
+    if (rc != CONCUR_OK || batch == 0) return rc;
+    // small batches plan in-kernel and need no plan call; larger ones need the matching one
+    const bool planned = h->planned_batch == batch && h->planned_stride == block_table_stride &&
+                         h->planned_lens == seq_lens;
+    if (batch > kSelfPlanBatch && !planned) return CONCUR_ERR_INVALID_ARG;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok()) return CONCUR_ERR_CUDA;
+    DecodeParams p = {};
+    fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
+                block_table_stride);
+    return enqueue(h, p, static_cast<cudaStream_t>(cuda_stream), planned);
+}
+
 int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                      const int32_t* block_table, int32_t* seq_lens, int32_t batch, int32_t num_pages,
                      int32_t block_table_stride, void* cuda_stream) {
-    if (!h) return CONCUR_ERR_INVALID_ARG;
+    return concur_kv_append_layer(h, k_new, v_new, k_pages, v_pages, block_table, seq_lens, batch, num_pages,
+                                  block_table_stride, 1, cuda_stream);
+}
+
+int concur_kv_append_layer(concur_attn_t* h, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
+                           const int32_t* block_table, int32_t* seq_lens, int32_t batch, int32_t num_pages,
+                           int32_t block_table_stride, int32_t advance, void* cuda_stream) {
+    if (!h || (advance != 0 && advance != 1)) return CONCUR_ERR_INVALID_ARG;
     if (batch < 0 || num_pages < 1 || block_table_stride < 1) return CONCUR_ERR_INVALID_ARG;
     if (batch > h->cfg.max_batch || block_table_stride > h->cfg.max_pages_per_seq) return CONCUR_ERR_TOO_LARGE;
     if ((int64_t)num_pages * h->cfg.num_kv_heads * h->cfg.page_size >= (int64_t)1 << 31) return CONCUR_ERR_TOO_LARGE;
@@ -242,7 +312,7 @@ int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, voi
     const int32_t shift = P == 16 ? 4 : (P == 32 ? 5 : (P == 64 ? 6 : 7));
     if (launch_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
                       reinterpret_cast<int32_t*>(h->ws + h->lay.hdr), batch, num_pages, block_table_stride, P,
-                      shift, h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0, h->cfg.num_kv_heads,
+                      shift, h->cfg.kv_layout == CONCUR_KV_TOKEN_MAJOR ? 1 : 0, h->cfg.num_kv_heads, advance,
                       static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return CONCUR_ERR_CUDA;
     return CONCUR_OK;
@@ -316,12 +386,13 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
     p.fuse_combine = 0;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    h->planned_batch = -1;
     if (launch_plan_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if (h->ev_before && cudaEventRecord(h->ev_before, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if ((h->prefix_kernel == 1 ? launch_prefix_mma(p, c, stream) : launch_prefix_tc(p, c, stream)) != cudaSuccess)
         return CONCUR_ERR_CUDA;
     if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
-    cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream);
+    cudaError_t e = h->kernel == 1 ? launch_partial_scalar(p, stream) : launch_partial_mma(p, stream, &h->maps);
     if (e != cudaSuccess) return CONCUR_ERR_CUDA;
     if (launch_combine_cascade(p, c, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     return CONCUR_OK;
@@ -347,6 +418,7 @@ int concur_prefill_attn(concur_attn_t* h, const void* q, const void* k_pages, co
     f.q_start = q_start;
     f.total_q = total_q;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    h->planned_batch = -1;
     if (h->ev_before && cudaEventRecord(h->ev_before, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if (launch_prefill_tc(p, f, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
@@ -415,6 +487,13 @@ int concur_attn_status(concur_attn_t* h, void* cuda_stream, uint32_t* flags) {
         cudaGetLastError();
         return CONCUR_ERR_CUDA;
     }
+    // A kernel in which a wait gave up may have left the range counter and the units' ticket counters
+    // half-way (only complete launches put them back to zero): start over.
+    if ((v & kFlagWaitLimit) &&
+        (cudaMemsetAsync(h->ws, 0, h->lay.part_lse, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess)) {
+        cudaGetLastError();
+        return CONCUR_ERR_CUDA;
+    }
     *flags = v;
     return CONCUR_OK;
 }
@@ -449,6 +528,12 @@ int concur_attn_set_option(concur_attn_t* h, int32_t key, int64_t value) {
         case CONCUR_OPT_SMALL_PAGE_COPY:
             if (value > 1) return CONCUR_ERR_INVALID_ARG;
             h->small_page_copy = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_OVERLAP_CALLS:
+            if (value > 1) return CONCUR_ERR_INVALID_ARG;
+            h->overlap_calls = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_WAIT_LIMIT_NS:
+            if (value > 60000000000ll) return CONCUR_ERR_INVALID_ARG;
+            h->wait_limit_ns = value > 0 ? value : 2000000000ll; return CONCUR_OK;
         case CONCUR_OPT_EVENT_BEFORE_PARTIAL:
             h->ev_before = reinterpret_cast<cudaEvent_t>(static_cast<uintptr_t>(value)); return CONCUR_OK;
         case CONCUR_OPT_EVENT_AFTER_PARTIAL:

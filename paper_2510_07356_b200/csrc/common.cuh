@@ -27,6 +27,8 @@ enum HeaderWord : int {
     kHdrClaim = 2,        // next range to hand out (atomic)
     kHdrStatus = 3,       // sticky CONCUR_FLAG_* bits
     kHdrWaitSite = 4,     // which wait gave up first (diagnostic; 0 = none)
+    kHdrClaimSelf = 5,    // launches without a plan kernel: ranges claimed so far beyond one per CTA; the
+                          // launch's last claim puts it back to 0
     kHdrWords = 64
 };
 
@@ -61,6 +63,13 @@ struct DecodeParams {
     int32_t max_ranges;       // capacity of range_start / partial slots
     int32_t fuse_combine;     // tensor-core kernel: 1 = the last partial of a unit merges it in-kernel
     int32_t claim_ahead;      // tiles before a range's end at which the next range is claimed
+    int32_t no_plan_launch;   // tensor-core partial kernel: 1 = no plan kernel ran before this launch.  Ranges are
+                              // claimed from kHdrClaimSelf, which the launch's last claim resets; the CTA that merges
+                              // a unit puts the unit's ticket counter back to 0; CTA 0 writes the results of empty
+                              // sequences, the bad-length flag, W, R and the range table
+    int32_t overlap_next;     // 1 = let the next launch on the stream (if it allows programmatic launch) start
+                              // while this one drains
+    int64_t wait_limit_ns;    // tensor-core partial kernel: after this long a role's wait gives up (flag, abort, return)
     // workspace
     int32_t* hdr;             // [kHdrWords]
     int32_t* tiles_prefix;    // [batch + 1] exclusive prefix of per-sequence tile counts
@@ -206,7 +215,8 @@ __device__ __forceinline__ Segment segment_at(const int32_t* __restrict__ prefix
 // Host-side launchers (each enqueues on `stream` and returns the launch status).
 cudaError_t launch_plan(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_partial_scalar(const DecodeParams& p, cudaStream_t stream);
-cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream);
+struct RowsMapCache;
+cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream, RowsMapCache* maps = nullptr);
 cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_plan_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
@@ -217,6 +227,6 @@ int partial_scalar_ctas_per_sm();
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                           const int32_t* block_table, int32_t* seq_lens, int32_t* hdr, int32_t batch,
                           int32_t num_pages, int32_t bt_stride, int32_t page_size, int32_t page_shift,
-                          int32_t token_major, int32_t hkv, cudaStream_t stream);
+                          int32_t token_major, int32_t hkv, int32_t advance, cudaStream_t stream);
 
 }  // namespace concur

@@ -28,6 +28,8 @@
 // copies it has in flight.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tensor_map.cuh"
@@ -85,11 +87,8 @@ static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
 
 }  // namespace
 
-__global__ void __launch_bounds__(kThreads, 1)
-partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+__device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CUtensorMap& map_k,
+                                                 const CUtensorMap& map_v, uint8_t* smem) {
     const uint32_t smem_base = smem_u32(smem);
     float* merge_o = reinterpret_cast<float*>(smem + Smem::kMergeOff);
     float* merge_ml = reinterpret_cast<float*>(smem + Smem::kMlOff);
@@ -119,6 +118,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     // the same swizzled layout; a tile's barrier then takes one arrival per copying lane (when that
     // lane's copies have landed) next to the producer's own.
     const bool lane_copy = p.lane_copy != 0;
+    const uint64_t wait_ns = (uint64_t)p.wait_limit_ns;       // the roles' waits; the drain of copies in flight keeps 2 s
     constexpr uint32_t kCopyLanes = (1 + kCopyWarps) * 32;
 
     if (tid == 0) {
@@ -153,6 +153,9 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     const bool self_plan = cached && p.tok_offset == nullptr && !p.all_partial;
     bool plan_seen = !self_plan;
     int32_t W, R;
+    // (opt-in) the next launch on the stream may begin while this one drains: its CTAs take the SMs this
+    // launch's CTAs leave, fill their rings, and wait for this grid's end before their first claim or store
+    if (p.overlap_next) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (self_plan) {
         int32_t* scan_ws = reinterpret_cast<int32_t*>(smem + Smem::kScanOff);
         if (tid == 0) sm_prefix[0] = 0;
@@ -163,6 +166,9 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             if (b < p.batch) {
                 const int64_t nn = p.seq_lens[b];
                 const int32_t n = (int32_t)(nn < 0 ? 0 : (nn > max_len ? max_len : nn));
+                // without a plan kernel, CTA 0 is the one that reports a length outside [0, stride * P]
+                if (p.no_plan_launch && blockIdx.x == 0 && n != nn)
+                    atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagBadLen);
                 sm_len[b] = n;
                 v = (n + kTile - 1) / kTile;
             }
@@ -210,6 +216,18 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         }
     };
     const int32_t* prefix = cached ? sm_prefix : p.tiles_prefix;
+    // The next range nobody has.  After a plan kernel the counter starts at the grid size (CTA i began on
+    // range i).  Without one there is nobody to reset a counter, so: with no more ranges than CTAs
+    // there is nothing to claim and no counter is touched; otherwise the counter counts this launch's
+    // claims from 0, and since every range that is streamed claims exactly once, the claim that draws
+    // R - 1 is the launch's last and puts the counter back to 0 for the next launch.
+    auto claim_range = [&]() -> int32_t {
+        if (!p.no_plan_launch) return atomicAdd(p.hdr + kHdrClaim, 1);
+        if (R <= (int32_t)gridDim.x) return R;
+        const int32_t c = atomicAdd(p.hdr + kHdrClaimSelf, 1);
+        if (c == R - 1) atomicExch(p.hdr + kHdrClaimSelf, 0);
+        return (int32_t)gridDim.x + c;
+    };
 
     // lane_copy: one instruction moves two 256-byte rows (lanes 0-15 the even row, 16-31 the odd
     // one), 16-byte piece c16 of a row each.  In a box's [half][row][128 B] layout with the
@@ -245,7 +263,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         const int w = warp - kCopyWarp0 + 1;
         for (uint32_t it = 0;; ++it) {
             const int s = it % kStages;
-            if (!mbar_wait(sched(s), (it / kStages) & 1u, abort_flag)) {
+            if (!mbar_wait(sched(s), (it / kStages) & 1u, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 10);
                 return;
             }
@@ -293,7 +311,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                     if (!claimed && x1 - (unit_start + t) <= p.claim_ahead &&
                         (plan_seen || unit_start + t - x0 >= kStages || unit_start + t == x1 - 1)) {
                         see_plan();
-                        if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
+                        if (lane == 0) r_next = claim_range();
                         claimed = true;
                     }
                     const int32_t tok_abs = off + t * kTile;               // first token of the tile in its sequence
@@ -320,7 +338,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                     const int32_t page2 = __shfl_sync(0xffffffffu, my_page, 2);
                     const int32_t page3 = __shfl_sync(0xffffffffu, my_page, 3);
                     if (lane == 0) {
-                        ok = mbar_wait(empty(s), parity ^ 1u, abort_flag);
+                        ok = mbar_wait(empty(s), parity ^ 1u, abort_flag, wait_ns);
                         if (ok) {
                             StageMeta& m = meta[s];
                             m.b = sg.b; m.g = sg.g; m.slot = sg.slot; m.n_valid = n_valid;
@@ -363,7 +381,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             // its ticket here, so the loop always moves on to a range nobody else has.
             if (ok && !claimed) {
                 see_plan();
-                if (lane == 0) r_next = atomicAdd(p.hdr + kHdrClaim, 1);
+                if (lane == 0) r_next = claim_range();
                 claimed = true;
             }
             r = __shfl_sync(0xffffffffu, r_next, 0);
@@ -373,7 +391,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 // tell the consumers that there is no more work
                 const int s = it % kStages;
                 const uint32_t parity = (it / kStages) & 1u;
-                ok = mbar_wait(empty(s), parity ^ 1u, abort_flag);
+                ok = mbar_wait(empty(s), parity ^ 1u, abort_flag, wait_ns);
                 if (ok) {
                     meta[s].n_valid = 0;
                     mbar_arrive_n(full_k(s), lane_copy ? 1 + kCopyLanes : 1);
@@ -403,8 +421,30 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
         // with a running maximum, 4 dims per lane, all 8 heads in flight at once.
         const float ninf_c = -INFINITY;
         see_plan();
+        if (p.no_plan_launch && blockIdx.x == 0) {
+            // What the plan kernel would have written besides its tables: the results of sequences without
+            // cached tokens, and (when this launch planned for itself) W, R and the range boundaries, which
+            // the plan query reads back.
+            if (self_plan) {
+                if (lane == 0) { p.hdr[kHdrTotalTiles] = W; p.hdr[kHdrNumRanges] = R; }
+                for (int32_t r = lane; r <= R; r += 32) p.range_start[r] = R > 0 ? range_begin(W, R, r) : 0;
+            }
+            for (int32_t b0 = 0; b0 < p.batch; b0 += 32) {
+                const int32_t b = b0 + lane;
+                int32_t n = 1;
+                if (b < p.batch) n = cached ? sm_len[b] : max(0, p.seq_lens[b]);
+                unsigned empties = __ballot_sync(0xffffffffu, n == 0);
+                while (empties) {
+                    const int e = b0 + (__ffs(empties) - 1);
+                    empties &= empties - 1;
+                    uint4* o = reinterpret_cast<uint4*>(p.out + (int64_t)e * p.hq * kD);
+                    for (int i = lane; i < p.hq * kD / 8; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+                    for (int i = lane; i < p.hq; i += 32) p.lse[(int64_t)e * p.hq + i] = ninf_c;
+                }
+            }
+        }
         for (uint32_t jobn = 0;; ++jobn) {
-            if (!mbar_wait(job_ready, jobn & 1u, abort_flag)) {
+            if (!mbar_wait(job_ready, jobn & 1u, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 8);
                 return;
             }
@@ -423,6 +463,8 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             const int32_t r_hi = range_of(W, R, ju + jt - 1);
             const int32_t splits = r_hi - r_lo + 1;
             if (ticket != splits - 1) continue;
+            // every ticket of this unit has been drawn: the counter goes back to 0 for the next launch
+            if (lane == 0) p.unit_done[jb * p.hkv + jg] = 0;
             // the unit's segment in range r is that range's first (slot 2r) unless the range
             // began before the unit did, which can only be the case for r_lo
             const int32_t slot_lo = 2 * r_lo + (range_begin(W, R, r_lo) < ju ? 1 : 0);
@@ -494,7 +536,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     for (uint32_t it = 0;; ++it) {
         const int s = it % kStages;
         const uint32_t parity = (it / kStages) & 1u;
-        if (!mbar_wait(full_k(s), parity, abort_flag)) {
+        if (!mbar_wait(full_k(s), parity, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 2);
                 return;
         }
@@ -504,12 +546,12 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             // All consumer threads meet first, so that no exit arrival can be counted into a
             // job phase that thread 0 (which may still be waiting to post it) has not joined.
             mbar_arrive(merge_bar0);
-            if (!mbar_wait(merge_bar0, merges & 1u, abort_flag)) {
+            if (!mbar_wait(merge_bar0, merges & 1u, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 9);
                 return;
             }
             if (tid == 0) {
-                if (mbar_wait(job_taken, (jobs & 1u) ^ 1u, abort_flag)) job_s->exit = 1;
+                if (mbar_wait(job_taken, (jobs & 1u) ^ 1u, abort_flag, wait_ns)) job_s->exit = 1;
                 else wait_failed(p, abort_flag, 7);
             }
             mbar_arrive(job_ready);
@@ -569,7 +611,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
             const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01));
             const uint32_t pb1 = movmatrix_trans(pack_bf16(p10, p11));
 
-            if (!mbar_wait(full_v(s), parity, abort_flag)) {
+            if (!mbar_wait(full_v(s), parity, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 3);
                 return;
             }
@@ -622,7 +664,7 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 ml[0] = m0; ml[1] = l0; ml[2] = m1; ml[3] = l1;
             }
             mbar_arrive(merge_bar0);
-            if (!mbar_wait(merge_bar0, merges & 1u, abort_flag)) {
+            if (!mbar_wait(merge_bar0, merges & 1u, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 4);
                 return;
             }
@@ -671,14 +713,14 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
                 }
             }
             mbar_arrive(merge_bar1);
-            if (!mbar_wait(merge_bar1, merges & 1u, abort_flag)) {
+            if (!mbar_wait(merge_bar1, merges & 1u, abort_flag, wait_ns)) {
                 if (lane == 0) wait_failed(p, abort_flag, 5);
                 return;
             }
             if (mt.slot >= 0 && p.fuse_combine) {
                 // hand the finished partial to the combiner warp; nobody here waits for it
                 if (tid == 0) {
-                    if (!mbar_wait(job_taken, (jobs & 1u) ^ 1u, abort_flag)) wait_failed(p, abort_flag, 6);
+                    if (!mbar_wait(job_taken, (jobs & 1u) ^ 1u, abort_flag, wait_ns)) wait_failed(p, abort_flag, 6);
                     job_s->b = mt.b; job_s->g = mt.g; job_s->unit_start = mt.unit_start;
                     job_s->tiles_b = mt.tiles_b; job_s->exit = 0;
                 }
@@ -690,29 +732,46 @@ partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
     }
 }
 
+__global__ void __launch_bounds__(kThreads, 1)
+partial_mma_kernel(DecodeParams p, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    partial_mma_body(p, map_k, map_v, smem);
+}
+
 // ------------------------------------------------------------------ host side
 
-cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
-    static bool attr_set[64] = {};
+cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream, RowsMapCache* maps) {
+    // the attribute is a property of the function on a device: setting it twice (two threads racing
+    // through here) is harmless, so an atomic flag per device is all the ordering this needs
+    static std::atomic<bool> attr_set[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 64 && !attr_set[dev]) {
+    if (dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
         e = cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
-    } else if (dev >= 64) {
-        e = cudaFuncSetAttribute(partial_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
+        if (dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
-    CUtensorMap map_k, map_v;
     // one box {64, rows of a box, 2} = the part of one (page, KV head) chunk that belongs to a tile
     const uint64_t pool_rows = (uint64_t)p.num_pages * p.page_size * (p.token_major ? 1 : p.hkv);
     const uint32_t planes = p.token_major ? 2 * p.hkv : 2;
-    if (!make_rows_map(&map_k, p.k_pages, pool_rows, p.box_rows, 2, planes) ||
-        !make_rows_map(&map_v, p.v_pages, pool_rows, p.box_rows, 2, planes))
+    CUtensorMap local_k, local_v;
+    const CUtensorMap *mk = &local_k, *mv = &local_v;
+    if (maps) {
+        mk = maps->get(p.k_pages, pool_rows, p.box_rows, 2, planes);
+        mv = maps->get(p.v_pages, pool_rows, p.box_rows, 2, planes);
+        if (!mk || !mv) return cudaErrorInvalidValue;
+    } else if (!make_rows_map(&local_k, p.k_pages, pool_rows, p.box_rows, 2, planes) ||
+               !make_rows_map(&local_v, p.v_pages, pool_rows, p.box_rows, 2, planes)) {
         return cudaErrorInvalidValue;
-    // programmatic dependent launch: the prologue (barrier set-up) may overlap the plan kernel
+    }
+    // Programmatic dependent launch: the kernel may start before the kernel ahead of it on the stream
+    // has finished, if that kernel allows it.  After this library's plan kernel that is always wanted
+    // (the prologue and the first tiles overlap the plan).  Without a plan kernel the kernel ahead is
+    // the caller's, and this kernel reads seq_lens, q and the pools before it waits: only a caller who
+    // has said that those are not that kernel's outputs gets the early start.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.grid_ctas);
     cfg.blockDim = dim3(kThreads);
@@ -722,8 +781,8 @@ cudaError_t launch_partial_mma(const DecodeParams& p, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, partial_mma_kernel, p, map_k, map_v);
+    cfg.numAttrs = (!p.no_plan_launch || p.overlap_next) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, partial_mma_kernel, p, *mk, *mv);
 }
 
 }  // namespace concur

@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DecodeParams p) {
         }
         // sequences without cached tokens get their result here (out = 0, lse = -inf): the
         // warp that found one writes it
-        unsigned empties = __ballot_sync(0xffffffffu, b < p.batch && tiles == 0);
+        unsigned empties = __ballot_sync(0xffffffffu, p.out != nullptr && b < p.batch && tiles == 0);
         while (empties) {
             const int e = base + warp * 32 + (__ffs(empties) - 1);
             empties &= empties - 1;

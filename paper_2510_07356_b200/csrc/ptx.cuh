@@ -39,17 +39,23 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait.  Returns false if the limit ran out or another warp raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t* abort_flag) {
+// Bounded wait.  Returns false if the limit ran out or another warp raised the abort flag.  A poll may
+// itself block for a hardware-defined while, so time is measured, not counted -- but lazily, because
+// most waits end within a few polls and reading the timer costs as much as several of them: the clock
+// is first read at poll 256 (for limits below a millisecond: at the second poll) and the limit counts
+// from that reading.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
+    const uint32_t every = limit_ns < 1000000ull ? 0u : 255u;
     uint64_t t0 = 0;
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0) {
+        if ((it & every) == 0) {
             if (*abort_flag) return false;
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
 }

@@ -117,6 +117,7 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.max_ranges = kStaticMaxRanges;
     p.fuse_combine = 1;
     p.claim_ahead = 1 << 20;
+    p.wait_limit_ns = 2000000000ll;
     // the plan kernel rewrites the tile count, the range count, the claim counter and the
     // per-unit counters at the start of every call, and every partial slot is written before
     // it is read, so nothing of the previous call's contents has to be cleared here

@@ -45,4 +45,33 @@ inline bool make_rows_map(CUtensorMap* map, const void* base, uint64_t rows, uin
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The maps of recent (base address, shape) combinations, so that a caller that alternates between a few
+// pools -- the layers of a model, one decode step after the other -- encodes each map once instead of
+// on every call.  A map holds nothing but what the key holds, so a hit is exact.  Not thread-safe:
+// it lives in a handle, and calls on one handle are ordered by the caller.
+struct RowsMapCache {
+    static constexpr int kEntries = 160;          // K and V pools of 64 layers, and some
+    struct Entry {
+        const void* base = nullptr;
+        uint64_t rows = 0;
+        uint32_t box_rows = 0, box_planes = 0, planes = 0;
+        CUtensorMap map;
+    };
+    Entry e[kEntries];
+    int used = 0, next = 0;
+
+    const CUtensorMap* get(const void* base, uint64_t rows, uint32_t box_rows, uint32_t box_planes, uint32_t planes) {
+        for (int i = 0; i < used; ++i)
+            if (e[i].base == base && e[i].rows == rows && e[i].box_rows == box_rows && e[i].box_planes == box_planes &&
+                e[i].planes == planes)
+                return &e[i].map;
+        Entry& x = e[next];
+        if (!make_rows_map(&x.map, base, rows, box_rows, box_planes, planes)) { x.base = nullptr; return nullptr; }
+        x.base = base; x.rows = rows; x.box_rows = box_rows; x.box_planes = box_planes; x.planes = planes;
+        next = (next + 1) % kEntries;
+        if (used < kEntries) ++used;
+        return &x.map;
+    }
+};
+
 }  // namespace concur

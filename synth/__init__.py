@@ -166,7 +166,9 @@ def _normal_bf16(shape, std, gen, device, chunk_elems=1 << 28):
 
 
 def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = None,
-                  spare_tokens: int = 0) -> Workload:
+                  spare_tokens: int = 0, value_seed: int | None = None) -> Workload:
+    """`value_seed` (default: the spec's seed) seeds q, K and V only: workloads that differ in it alone
+    share lengths and block table and hold different values -- the layers of one model."""
     if isinstance(spec, str):
         spec = SPECS[spec]
     device = torch.device(device)
@@ -176,7 +178,7 @@ def make_workload(spec: Spec | str, device="cpu", table_stride: int | None = Non
 
     def gen(stream):
         g = torch.Generator(device=device)
-        g.manual_seed(spec.seed * 1000 + stream)
+        g.manual_seed((spec.seed if value_seed is None else value_seed) * 1000 + stream)
         return g
 
     q = _normal_bf16((spec.batch, Hq, D), spec.q_std, gen(3), device)

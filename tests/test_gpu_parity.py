@@ -328,3 +328,30 @@ def test_repeated_calls_on_one_handle_are_identical(P):
     assert_parity(first[2], first[3], ref_out, ref_lse, "small after big")
     assert attn.status() == 0
     attn.close()
+
+
+def test_a_wait_that_runs_out_returns_with_the_flag_and_leaves_the_handle_usable(P):
+    # One CTA streams a whole 16,384-token sequence in two ranges that cut no unit, so its combiner
+    # warp has nothing to merge and waits for a job from the kernel's start to its end, hundreds of
+    # microseconds.  With the roles' wait limit set to 20 microseconds that wait gives up: the
+    # kernel must still end by itself, report CONCUR_FLAG_WAIT_LIMIT, and fault nothing; with the
+    # default limit back, the same handle then computes the right result.
+    spec = synth.tiny_spec("waitlimit", (16384,), 64, 1300)
+    w = synth.make_workload(spec, "cuda:0")
+    attn = P.DecodeAttention(64, 1, w.block_table.shape[1], 0)
+    attn.set_option(P.CONCUR_OPT_GRID_CTAS, 1)
+    attn.set_option(P.CONCUR_OPT_NUM_RANGES, 2)
+    attn.set_option(P.CONCUR_OPT_WAIT_LIMIT_NS, 20_000)
+    out, lse = attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
+    torch.cuda.synchronize()
+    assert attn.status() & P.CONCUR_FLAG_WAIT_LIMIT
+    assert attn.status() == 0                                   # reading the flags clears them
+    attn.set_option(P.CONCUR_OPT_WAIT_LIMIT_NS, 0)              # the default again
+    ref_out, ref_lse = oracle_sequences(to_host(w))
+    for grid in (1, 0):
+        attn.set_option(P.CONCUR_OPT_GRID_CTAS, grid)
+        out, lse = attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
+        torch.cuda.synchronize()
+        assert attn.status() == 0
+        assert_parity(out, lse, ref_out, ref_lse, f"after a wait limit, grid {grid}")
+    attn.close()

@@ -52,6 +52,42 @@ def test_reference_append_is_concatenation():
     assert (k != k1).any(axis=3).sum() == 2 * hkv          # only sequences 2 and 3 were written
 
 
+def test_reference_append_for_the_further_layers_of_a_step():
+    # two layers, one set of lengths: the first layer's append opens the slot and advances, the second
+    # layer's append (advance=False) fills the same slot of its own pools; after T steps both layers hold
+    # their own concatenation and the lengths have grown by T, not 2 T
+    rng = np.random.default_rng(5)
+    P, hkv, D, steps, B = 4, 2, 8, 5, 3
+    lens0 = np.array([0, 3, 8], dtype=np.int32)
+    pages_per = -(-(lens0 + steps) // P)
+    table = np.full((B, pages_per.max()), -1, dtype=np.int32)
+    perm = rng.permutation(int(pages_per.sum()))
+    at = 0
+    for b, n in enumerate(pages_per):
+        table[b, :n] = perm[at:at + n]; at += n
+    pools = [[rng.integers(0, 65536, size=(at, hkv, P, D)).astype(np.uint16) for _ in range(2)] for _ in range(2)]
+    before = [[x.copy() for x in layer] for layer in pools]
+    new = rng.integers(0, 65536, size=(steps, 2, 2, B, hkv, D)).astype(np.uint16)      # [step][layer][k|v]
+    lens = lens0.copy()
+    for s in range(steps):
+        kv_cache.kv_append(pools[0][0], pools[0][1], table, lens, new[s, 0, 0], new[s, 0, 1])
+        kv_cache.kv_append(pools[1][0], pools[1][1], table, lens, new[s, 1, 0], new[s, 1, 1], advance=False)
+        assert np.array_equal(lens, lens0 + s + 1)
+    for layer in range(2):
+        for kv in range(2):
+            for b in range(B):
+                got = kv_cache.gather_tokens(pools[layer][kv], table, b, int(lens[b]))
+                want = np.concatenate([kv_cache.gather_tokens(before[layer][kv], table, b, int(lens0[b])),
+                                       new[:, layer, kv, b]])
+                assert np.array_equal(got, want)
+            assert (pools[layer][kv] != before[layer][kv]).any(axis=3).sum() == steps * B * hkv
+    # a sequence with no token yet has no slot for a further layer to fill: nothing moves
+    k, v = pools[1][0].copy(), pools[1][1].copy()
+    zero = np.zeros(B, dtype=np.int32)
+    kv_cache.kv_append(k, v, table, zero, new[0, 1, 0], new[0, 1, 1], advance=False)
+    assert np.array_equal(k, pools[1][0]) and np.array_equal(zero, np.zeros(B, dtype=np.int32))
+
+
 @pytest.fixture(scope="module")
 def P():
     import __graft_entry__
