@@ -112,6 +112,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// 2^x on the FMA and integer pipes, for x <= 127 (anything below -126, -inf included, gives ~2^-126):
+// x = n + f with n the nearest integer (the 1.5 * 2^23 trick leaves n in the low mantissa bits) and
+// |f| <= 1/2; 2^f by a degree-4 polynomial (relative error 4e-5, far inside what a bf16 probability
+// keeps); n goes into the exponent field by an integer add.  Used for a share of a softmax tile's
+// exponentials so that they do not all queue on the special-function unit (4 lanes per clock and SM
+// sub-partition against 32 for an FMA).
+__device__ __forceinline__ float exp2_fma(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;                       // 1.5 * 2^23: rounds x to an integer
+    const float f = x - (t - 12582912.f);
+    float r = fmaf(f, 0.0096181291f, 0.0555041087f);
+    r = fmaf(r, f, 0.2402265070f);
+    r = fmaf(r, f, 0.6931471806f);
+    r = fmaf(r, f, 1.0f);
+    return __uint_as_float(__float_as_uint(r) + (__float_as_uint(t) << 23));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
