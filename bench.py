@@ -101,7 +101,7 @@ class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index):
         self.index = index
@@ -138,7 +138,7 @@ class ClockSampler:
         rows = [l for (t, l) in self.lines if (t0 is None or t >= t0 - 0.05) and (t1 is None or t <= t1 + 0.1)]
         if not rows:
             rows = [l for _, l in self.lines]
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, watts = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             parts = [x.strip() for x in r.split(",")]
@@ -151,8 +151,13 @@ class ClockSampler:
             for n, v in zip(names, parts[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
+            try:
+                watts.append(float(parts[6]))
+            except (IndexError, ValueError):
+                pass
         return {"sm_mhz": statistics.median(sm) if sm else None,
-                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm),
+                "power_w": statistics.median(watts) if watts else None}
 
 
 class L2Flush:
@@ -1035,32 +1040,54 @@ def main():
     # ---- the same step back to back for about two seconds: what the power cap leaves of the burst figure
     sustained = None
     if flush_buf is None and args.sustained_seconds > 0:
-        def back_to_back(fn, one_ms, seconds):
+        def back_to_back(fn, one_ms, seconds, stamps=None):
             chunk = max(10, int(0.1 / max(one_ms * 1e-3, 1e-6)))           # about 0.1 s of calls per event pair
             marks, t_end = [], time.time() + seconds
             while time.time() < t_end:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                t_a = time.time()
                 e0.record(stream)
                 for _ in range(chunk):
                     fn()
                 e1.record(stream)
                 e1.synchronize()
                 marks.append(e0.elapsed_time(e1) / chunk)
+                if stamps is not None:
+                    stamps.append((0.5 * (t_a + time.time()), marks[-1]))
             tail = marks[len(marks) // 2:]                                 # the second half: clocks have settled
             return sum(tail) / len(tail), marks[0], chunk * len(marks)
+
+        def by_clock(stamps, sampler_lines):
+            """Chunks of the sustained run grouped by the SM clock sampled nearest to them: how the step
+            time moves with the clock the power cap leaves (no clock is ever set from here)."""
+            pts = []
+            for t, l in sampler_lines:
+                try:
+                    pts.append((t, float(l.split(",")[0])))
+                except ValueError:
+                    pass
+            if not pts:
+                return None
+            bins = {}
+            for t, ms in stamps:
+                mhz = min(pts, key=lambda q: abs(q[0] - t))[1]
+                bins.setdefault(mhz, []).append(ms)
+            return [{"sm_mhz": k, "chunks": len(v), "ms_per_step": sum(v) / len(v), "ms_x_ghz": sum(v) / len(v) * k / 1e3}
+                    for k, v in sorted(bins.items())]
 
         sampler2 = ClockSampler(gpu_id)
         if rank == 0:
             sampler2.start()
             time.sleep(0.2)
         t_s0 = time.time()
-        sus_ms, first_ms, n_steps = back_to_back(step, ms_per_step, args.sustained_seconds)
+        stamps = []
+        sus_ms, first_ms, n_steps = back_to_back(step, ms_per_step, args.sustained_seconds, stamps)
         t_s1 = time.time()
         sus_clocks = sampler2.stop(t_s0, t_s1) if rank == 0 else None
         sus_ms = over_ranks([sus_ms], "max", dev)[0]
         sustained = {"ms_per_step": sus_ms, "value": job_bytes / (sus_ms * 1e-3) / 1e9, "unit": UNIT,
                      "seconds": args.sustained_seconds, "steps": n_steps, "first_chunk_ms_per_step": first_ms,
-                     "clocks": sus_clocks,
+                     "clocks": sus_clocks, "by_clock": by_clock(stamps, sampler2.lines) if rank == 0 else None,
                      "what": "steps back to back; mean of the second half of the interval"}
         # the read-only stream under the same regime, so that the two can be compared like for like
         pool_b = w.k_pages.numel() * 2 + w.v_pages.numel() * 2
@@ -1070,8 +1097,17 @@ def main():
             bench_probe.read_probe(w.k_pages, w.k_pages.numel() * 2, chk_s[0:1], 0, stream.cuda_stream)
             bench_probe.read_probe(w.v_pages, w.v_pages.numel() * 2, chk_s[1:2], 0, stream.cuda_stream)
 
-        probe_ms, _, _ = back_to_back(probe_s, ms_per_step, args.sustained_seconds / 2)
+        sampler3 = ClockSampler(gpu_id)
+        if rank == 0:
+            sampler3.start()
+            time.sleep(0.2)
+        stamps_p = []
+        t_p0 = time.time()
+        probe_ms, _, _ = back_to_back(probe_s, ms_per_step, args.sustained_seconds / 2, stamps_p)
+        probe_clocks = sampler3.stop(t_p0, time.time()) if rank == 0 else None
         sustained["read_stream_gbs"] = pool_b / (probe_ms * 1e-3) / 1e9
+        sustained["read_stream_clocks"] = probe_clocks
+        sustained["read_stream_by_clock"] = by_clock(stamps_p, sampler3.lines) if rank == 0 else None
 
     # ---- yardstick: a plain read-only stream over the same two pools (only where they are well above L2)
     read_stream = None

@@ -36,8 +36,18 @@
  * result (they may hold anything, NaN included).
  *
  * Conventions: every function returns CONCUR_OK (0) or a negative concur_status_t; none
- * throws, aborts or prints.  No pointer is retained after a call returns.  The library
- * has no CPU fallback: without a CUDA device every call fails with CONCUR_ERR_CUDA.
+ * throws, aborts or prints.  No pointer is retained after a call returns (concur_attn_plan
+ * remembers the ADDRESS of seq_lens, to recognise the matching planned calls; it is never
+ * dereferenced on the host).  The library has no CPU fallback: without a CUDA device every call
+ * fails with CONCUR_ERR_CUDA.
+ *
+ * Host threads: a handle is not locked.  Calls on ONE handle (options, status and destroy included)
+ * must not run at the same time in two host threads; order them yourself.  Calls on DIFFERENT
+ * handles may run concurrently from different threads, and so may concur_attn_workspace_bytes,
+ * concur_attn_create and concur_attn_strerror: the library's only process-wide state is the
+ * one-time per-device set-up of its kernels, which is safe to race.  concur_decode_attn_static may be
+ * called from several threads as far as the host is concerned, but its calls share one device
+ * array per GPU and must not overlap ON THE GPU (see there).
  */
 #ifndef CONCUR_ATTN_H_
 #define CONCUR_ATTN_H_

@@ -14,6 +14,8 @@
 // cudaGetSymbolAddress (with that device current) and that pointer is what the kernels get.
 #include "../../include/concur_attn.h"
 
+#include <mutex>
+
 #include "common.cuh"
 
 using namespace concur;
@@ -42,10 +44,12 @@ struct DeviceSetup {
     int sm_count = 0;
 };
 DeviceSetup g_setup[kMaxDevices];
+std::mutex g_setup_mutex;      // two host threads may make a device's first call at the same time
 
 // Once per device, with that device current: resolve the array's device address.
 int setup_current_device(int dev, DeviceSetup** out) {
     if (dev < 0 || dev >= kMaxDevices) return CONCUR_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
     DeviceSetup& s = g_setup[dev];
     if (!s.ready) {
         void* ptr = nullptr;

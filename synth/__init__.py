@@ -58,6 +58,10 @@ SPECS = {
     "cfg3_b64_ctx16384_p64": Spec("cfg3_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563),
     # a quarter of cfg3 (same lengths, page size and values): small enough for profiler captures
     "cfg3q_b16_ctx16384_p64": Spec("cfg3q_b16_ctx16384_p64", 16, 64, ("const", 16384), q_std=0.5, seed=73563),
+    # config 3 with every sequence's pages in logical order, one sequence after the other (no shuffle): the
+    # same bytes as one linear stream per (sequence, head), to tell page placement from everything else
+    "cfg3c_b64_ctx16384_p64": Spec("cfg3c_b64_ctx16384_p64", 64, 64, ("const", 16384), permute_pages=False,
+                                   q_std=0.5, seed=73563),
     # config 3 with 40 query heads (group size 5): the geometry variant of the same workload
     "cfg3h40_b64_ctx16384_p64": Spec("cfg3h40_b64_ctx16384_p64", 64, 64, ("const", 16384), q_std=0.5, seed=73563,
                                      num_q_heads=40),
