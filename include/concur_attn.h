@@ -321,6 +321,30 @@ int concur_kv_append_layer(concur_attn_t* handle, const void* k_new, const void*
                            void* cuda_stream);
 
 /*
+ * concur_kv_append_layer(advance = 0) and concur_decode_attn in one: the K / V rows of every sequence's
+ * newest token -- position seq_lens[b] - 1, which the step's first append has already counted -- are
+ * passed in, used for the attention, and stored into their pool slot by the kernel itself.  One launch
+ * per layer instead of two (for up to 511 sequences), and, with CONCUR_OPT_OVERLAP_CALLS, layer after
+ * layer may overlap, which an append kernel between two attention kernels prevents.  The paper has no
+ * counterpart (it implies the generation loop, Sec. 3.3, and describes none of it).
+ *
+ *   k_new, v_new   device, bf16 [batch][Hkv][D], 16-byte aligned: rows of the token at seq_lens[b] - 1
+ *   k_pages, v_pages   as for concur_decode_attn, but WRITTEN: slot (seq_lens[b] - 1) % P of page
+ *                  block_table[b][(seq_lens[b] - 1) / P] receives the rows; whatever that slot held before
+ *                  is ignored
+ *   other arguments, result, asynchrony as for concur_decode_attn (seq_lens is only read)
+ *
+ * A sequence with seq_lens[b] = 0 has no newest token: nothing is stored, its result is that of an empty
+ * sequence.  A bad page id for the slot is flagged (CONCUR_FLAG_BAD_PAGE_ID) and nothing is stored.
+ * Needs the tensor-core kernel with the fused merge (the defaults): CONCUR_ERR_UNSUPPORTED otherwise.
+ */
+int concur_decode_attn_append(concur_attn_t* handle, const void* q, const void* k_new, const void* v_new,
+                              void* k_pages, void* v_pages, const int32_t* block_table,
+                              const int32_t* seq_lens, float scale, void* out, float* lse,
+                              int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                              void* cuda_stream);
+
+/*
  * The same step for callers whose tensors live in HOST memory (pinned memory gives
  * asynchronous copies).  Every pointer is a host pointer with the layouts above; the
  * library copies the inputs into device staging buffers that it owns (allocated on first

@@ -46,7 +46,7 @@ EXPORTS = (
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
     "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade", "concur_prefill_attn",
     "concur_curate", "concur_attn_plan", "concur_decode_attn_planned",
-    "concur_kv_append_layer",
+    "concur_kv_append_layer", "concur_decode_attn_append",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -110,6 +110,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_kv_append.restype = ctypes.c_int
     lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
+    lib.concur_decode_attn_append.restype = ctypes.c_int
+    lib.concur_decode_attn_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, vp]
     lib.concur_kv_append_layer.restype = ctypes.c_int
     lib.concur_kv_append_layer.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
@@ -279,6 +281,18 @@ def concur_kv_append_layer(handle, k_new, v_new, k_pages, v_pages, block_table, 
                                     int(advance), stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_kv_append_layer")
+    return rc
+
+
+def concur_decode_attn_append(handle, q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, scale, out, lse,
+                              batch, num_pages, block_table_stride, stream=0, check=True) -> int:
+    """Append (without advancing seq_lens) and attend in one launch: the newest token's rows come from
+    k_new / v_new and are stored into the pools by the attention kernel."""
+    rc = lib.concur_decode_attn_append(handle, _addr(q), _addr(k_new), _addr(v_new), _addr(k_pages), _addr(v_pages),
+                                       _addr(block_table), _addr(seq_lens), ctypes.c_float(scale), _addr(out),
+                                       _addr(lse), batch, num_pages, block_table_stride, stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_decode_attn_append")
     return rc
 
 

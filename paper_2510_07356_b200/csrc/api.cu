@@ -287,6 +287,26 @@ int concur_decode_attn_planned(concur_attn_t* h, const void* q, const void* k_pa
     return enqueue(h, p, static_cast<cudaStream_t>(cuda_stream), planned);
 }
 
+int concur_decode_attn_append(concur_attn_t* h, const void* q, const void* k_new, const void* v_new, void* k_pages,
+                              void* v_pages, const int32_t* block_table, const int32_t* seq_lens, float scale,
+                              void* out, float* lse, int32_t batch, int32_t num_pages, int32_t block_table_stride,
+                              void* cuda_stream) {
+    int rc = check_call(h, q, k_pages, v_pages, block_table, seq_lens, out, lse, batch, num_pages,
+                        block_table_stride, 16);
+    if (rc != CONCUR_OK || batch == 0) return rc;
+    if (!k_new || !v_new || !aligned(k_new, 16) || !aligned(v_new, 16)) return CONCUR_ERR_INVALID_ARG;
+    // only the tensor-core kernel with the merge fused takes its last token from outside the pools
+    if (h->kernel != 0 || !h->fuse_combine) return CONCUR_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->cfg.device);
+    if (!guard.ok()) return CONCUR_ERR_CUDA;
+    DecodeParams p = {};
+    fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
+                block_table_stride);
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    return enqueue(h, p, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int concur_kv_append(concur_attn_t* h, const void* k_new, const void* v_new, void* k_pages, void* v_pages,
                      const int32_t* block_table, int32_t* seq_lens, int32_t batch, int32_t num_pages,
                      int32_t block_table_stride, void* cuda_stream) {

@@ -78,6 +78,11 @@ struct DecodeParams {
     float* part_lse;          // [2 * max_ranges][kGroup]     base-2 log-sum-exp of each partial
     int32_t* unit_done;       // [batch * hkv] partial segments finished per (sequence, KV head) unit
     // shared-prefix (cascade) mode; both unset in the plain path
+    // fused append (tensor-core partial kernel): the K / V rows [batch][hkv][D] of each sequence's LAST token
+    // (position seq_lens[b] - 1) are taken from here instead of the pools, and stored into the pools by the
+    // CTA that streams the tile they belong to; both null in every other call
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
     const int32_t* tok_offset; // [batch] first token of each sequence that this pass covers (multiple of 64), or null
     int32_t all_partial;      // 1: every segment writes a partial into slot r + u (u = b * hkv + g)
 };

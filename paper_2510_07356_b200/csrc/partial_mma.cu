@@ -59,6 +59,10 @@ struct StageMeta {
     int32_t unit_start;    // flat tile index of the unit's first tile
     int32_t tiles_b;       // tiles of the whole unit
     int32_t page[4];       // small pages: pool pages of the tile's boxes (for the copy helpers)
+    int32_t new_row;       // fused append: row of the tile that is the sequence's new token, else -1
+    int32_t new_page;      // ... and the pool page its slot is in (-1: not to be stored, the page id was bad)
+    int32_t seg_new;       // fused append: 1 on a segment's first tile if the segment holds the unit's last tile
+    int32_t new_slot;      // fused append: slot of the new token inside new_page
 };
 
 // A finished partial segment handed from the consumer warps to the combiner warp.
@@ -333,6 +337,8 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                         if (lane == 0) atomicOr(reinterpret_cast<unsigned int*>(p.hdr + kHdrStatus), kFlagBadPage);
                         if (my_page < 0 || my_page >= p.num_pages) my_page = 0;
                     }
+                    // (fused append: was the page of the tile's last token among the clamped ones?)
+                    const bool new_page_bad = __shfl_sync(0xffffffffu, (int)bad, (n_valid - 1) >> p.box_shift) != 0;
                     const int32_t page0 = __shfl_sync(0xffffffffu, my_page, 0);
                     const int32_t page1 = __shfl_sync(0xffffffffu, my_page, 1);
                     const int32_t page2 = __shfl_sync(0xffffffffu, my_page, 2);
@@ -345,6 +351,14 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                             m.first = (t == sg.tile0); m.last = (t == sg.tile1 - 1);
                             m.unit_start = unit_start; m.tiles_b = sg.tiles_b;
                             m.page[0] = page0; m.page[1] = page1; m.page[2] = page2; m.page[3] = page3;
+                            // fused append: the sequence's last token sits in the unit's last tile
+                            const bool new_here = p.k_new != nullptr && t == sg.tiles_b - 1;
+                            const int32_t new_row = n_valid - 1;
+                            const int32_t new_pages[4] = {page0, page1, page2, page3};
+                            m.new_row = new_here ? new_row : -1;
+                            m.new_page = (new_here && !new_page_bad) ? new_pages[new_row >> p.box_shift] : -1;
+                            m.seg_new = (p.k_new != nullptr && sg.tile1 == sg.tiles_b) ? 1 : 0;
+                            m.new_slot = (tok_abs + new_row) & page_mask;
                             const uint32_t kdst = smem_base + s * kStageBytes;
                             const uint32_t vdst = kdst + kTileBytes;
                             const bool with_q = (t == sg.tile0);
@@ -532,6 +546,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
     #pragma unroll
     for (int i = 0; i < 8; ++i) { qf[i][0] = qf[i][1] = 0u; o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     uint32_t merges = 0, jobs = 0;
+    uint4 new_piece = make_uint4(0, 0, 0, 0);        // fused append: this lane's piece of the new token's K or V row
 
     for (uint32_t it = 0;; ++it) {
         const int s = it % kStages;
@@ -569,9 +584,35 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
             m0 = m1 = ninf; l0 = l1 = 0.f;
             #pragma unroll
             for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+            // fused append: this segment ends with the sequence's new token, whose rows come from k_new /
+            // v_new; fetch them now (lanes 0-15 a 16-byte piece of the K row each, lanes 16-31 of the V row)
+            // so that they are in registers by the time the last tile is
+            if (mt.seg_new)
+                new_piece = __ldg(reinterpret_cast<const uint4*>(
+                    (lane < 16 ? p.k_new : p.v_new) + ((int64_t)mt.b * p.hkv + mt.g) * kD + (lane & 15) * 8));
         }
         const int valid = mt.n_valid - tok0;          // valid tokens among this warp's 16
+        // fused append: is the new token one of this warp's rows of this tile?
+        const bool patch = mt.new_row >= tok0 && mt.new_row < tok0 + 16;
+        // where the 16-byte piece (lane & 15) of that row sits in a swizzled tile (relative to the tile's base)
+        const uint32_t patch_off = (uint32_t)(mt.new_row >> p.box_shift) * (uint32_t)P * kRowBytes +
+                                   (uint32_t)((lane & 15) >> 3) * half_stride + (uint32_t)(mt.new_row & (P - 1)) * 128u +
+                                   (uint32_t)((((lane & 15) & 7) ^ (mt.new_row & 7)) << 4);
         if (valid > 0) {
+            if (patch) {
+                // the pool's slot has not been written yet: put the K row where the copy left the slot's old
+                // contents, and store both rows into the pools for the steps to come
+                if (lane < 16)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(kbase + patch_off), "r"(new_piece.x),
+                                 "r"(new_piece.y), "r"(new_piece.z), "r"(new_piece.w) : "memory");
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (mt.new_page >= 0) {
+                    see_plan();
+                    __nv_bfloat16* pool = lane < 16 ? const_cast<__nv_bfloat16*>(p.k_pages) : const_cast<__nv_bfloat16*>(p.v_pages);
+                    *reinterpret_cast<uint4*>(pool + pool_elem(p, mt.new_page, mt.g, mt.new_slot) + (lane & 15) * 8) = new_piece;
+                }
+            }
             // ---- S^T = K . Q^T  (two accumulator chains to shorten the dependency)
             float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
             #pragma unroll
@@ -625,6 +666,13 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                                           (uint32_t)((c & 7) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0) : "memory");
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+            }
+            if (patch) {
+                if (lane >= 16)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(vbase + patch_off), "r"(new_piece.x),
+                                 "r"(new_piece.y), "r"(new_piece.z), "r"(new_piece.w) : "memory");
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }

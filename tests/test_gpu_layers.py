@@ -169,3 +169,83 @@ def test_append_layer_argument_errors(P):
     changed = (w.k_pages.view(torch.int16) != before.view(torch.int16)).any(dim=3).sum().item()
     assert changed == 8                                   # sequence 0's slot 4, all 8 KV heads
     attn.close()
+
+
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128])
+@pytest.mark.parametrize("token_major", [0, 1])
+@pytest.mark.parametrize("hkv,hq,ranges", [(8, 64, 0), (8, 64, 37), (2, 10, 0), (1, 8, 5)])
+def test_fused_append_equals_append_then_attend(P, page_size, token_major, hkv, hq, ranges):
+    # lengths already count the new token: it is the only token (1), the last slot of a page / tile (64, 128),
+    # the first slot of a fresh one (65, 129, 17), somewhere inside; 0 = no token at all
+    lens = (0, 1, 2, 16, 17, 63, 64, 65, 128, 129, 200, 1000, 1025, 4099)
+    spec = synth.tiny_spec(f"fa_p{page_size}", lens, page_size, 9800 + page_size + hkv, num_q_heads=hq, num_kv_heads=hkv)
+    w = synth.make_workload(spec, "cuda:0")
+    B = spec.batch
+    g = torch.Generator(device="cuda:0"); g.manual_seed(9900 + page_size)
+    kn = torch.randn((B, hkv, 128), generator=g, device="cuda:0").to(torch.bfloat16)
+    vn = torch.randn((B, hkv, 128), generator=g, device="cuda:0").to(torch.bfloat16)
+    # the slot of every sequence's newest token holds garbage until the call stores the rows there
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    for b, n in enumerate(lens):
+        if n:
+            page = int(w.table_host[b, (n - 1) // page_size])
+            w.k_pages[page, :, (n - 1) % page_size, :] = nan
+            w.v_pages[page, :, (n - 1) % page_size, :] = nan
+    # reference: the layer append of the write-path reference, then the attention oracle
+    k_ref, v_ref = bits(w.k_pages), bits(w.v_pages)
+    lens_ref = np.array(lens, dtype=np.int32)
+    kv_cache.kv_append(k_ref, v_ref, w.table_host, lens_ref, bits(kn), bits(vn), advance=False)
+    assert np.array_equal(lens_ref, np.array(lens, dtype=np.int32))
+    ref_out, ref_lse = oracle.decode_attn(w.q, k_ref, v_ref, w.table_host, lens_ref, w.scale)
+    k_dev, v_dev = w.k_pages, w.v_pages
+    if token_major:
+        k_dev = k_dev.permute(0, 2, 1, 3).contiguous(); v_dev = v_dev.permute(0, 2, 1, 3).contiguous()
+    attn = P.DecodeAttention(page_size, B, w.block_table.shape[1], 0, num_q_heads=hq, num_kv_heads=hkv,
+                             kv_layout=token_major)
+    attn.set_option(P.CONCUR_OPT_NUM_RANGES, ranges)
+    out = torch.full_like(w.q, 7.0)
+    lse = torch.full((B, hq), 7.0, dtype=torch.float32, device="cuda:0")
+    lens_dev = w.seq_lens.clone()
+    P.concur_decode_attn_append(attn.handle, w.q, kn, vn, k_dev, v_dev, w.block_table, lens_dev, w.scale, out, lse, B,
+                                w.num_pages, w.block_table.shape[1], torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert torch.equal(lens_dev, w.seq_lens)                      # lengths are only read
+    assert_parity(out, lse, ref_out, ref_lse, f"fused append p{page_size} tm{token_major} hkv{hkv} R{ranges}")
+    k_back = (k_dev.permute(0, 2, 1, 3) if token_major else k_dev).contiguous()
+    v_back = (v_dev.permute(0, 2, 1, 3) if token_major else v_dev).contiguous()
+    assert np.array_equal(bits(k_back), k_ref) and np.array_equal(bits(v_back), v_ref)   # byte for byte
+    # and the plain call on the pools as they are now gives the same again
+    out2, lse2 = attn(w.q, k_dev, v_dev, w.block_table, lens_dev, w.scale)
+    torch.cuda.synchronize()
+    assert_parity(out2, lse2, ref_out, ref_lse, "plain call after the fused one")
+    attn.close()
+
+
+def test_fused_append_needs_the_fused_tensor_core_path_and_flags_bad_pages(P):
+    B_ = P.binding
+    spec = synth.tiny_spec("fa_err", (70, 5), 64, 9950)
+    w = synth.make_workload(spec, "cuda:0")
+    kn = torch.zeros((2, 8, 128), dtype=torch.bfloat16, device="cuda:0")
+    out = torch.empty_like(w.q); lse = torch.empty((2, 64), dtype=torch.float32, device="cuda:0")
+    attn = P.DecodeAttention(64, 2, w.block_table.shape[1], 0)
+
+    def call(k_new=kn, table=w.block_table):
+        return B_.concur_decode_attn_append(attn.handle, w.q, k_new, kn, w.k_pages, w.v_pages, table, w.seq_lens, w.scale,
+                                            out, lse, 2, w.num_pages, w.block_table.shape[1], 0, check=False)
+    attn.set_option(P.CONCUR_OPT_KERNEL, 1)
+    assert call() == B_.CONCUR_ERR_UNSUPPORTED
+    attn.set_option(P.CONCUR_OPT_KERNEL, 0)
+    attn.set_option(P.CONCUR_OPT_FUSE_COMBINE, 0)
+    assert call() == B_.CONCUR_ERR_UNSUPPORTED
+    attn.set_option(P.CONCUR_OPT_FUSE_COMBINE, 1)
+    assert call(k_new=None) == B_.CONCUR_ERR_INVALID_ARG
+    # the page of sequence 1's newest token lies outside the pool: flagged, nothing stored, nothing faults
+    bad = w.block_table.clone(); bad[1, 0] = w.num_pages + 7
+    before = w.k_pages.clone()
+    assert call(table=bad) == B_.CONCUR_OK
+    torch.cuda.synchronize()
+    assert attn.status() & P.CONCUR_FLAG_BAD_PAGE_ID
+    changed = (w.k_pages.view(torch.int16) != before.view(torch.int16)).any(dim=3).sum().item()
+    assert changed <= 8                                           # at most sequence 0's slot, all 8 KV heads
+    attn.close()
