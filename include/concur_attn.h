@@ -77,6 +77,10 @@ typedef enum {
 #define CONCUR_FLAG_BAD_GROUP   8u  /* cascade step: group_start was not 0 <= g[0] <= g[1] <= ... <= batch;
                                        the call then shared nothing and computed the plain step          */
 
+#define CONCUR_FLAG_BOUNDS     16u  /* only from the checked build of the library (compiled with -DCONCUR_BOUNDS,
+                                       `python -m paper_2510_07356_b200.build --bounds`): an index the
+                                       kernels computed fell outside its buffer; the access was skipped    */
+
 /* Option keys for concur_attn_set_option (tuning and tests; defaults are chosen per call). */
 #define CONCUR_OPT_KERNEL      1    /* 0 = tensor-core partial kernel (default), 1 = scalar-FMA kernel */
 #define CONCUR_OPT_NUM_RANGES  2    /* force the number of split-KV ranges; 0 = heuristic              */

@@ -9,7 +9,11 @@ from __future__ import annotations
 import ctypes
 from pathlib import Path
 
-_LIB_PATH = Path(__file__).resolve().parent / "libconcur_attn.so"
+import os
+
+# CONCUR_ATTN_LIBRARY names another build of the same library to load instead -- the checked build
+# (libconcur_attn_bounds.so), whose kernels verify every index they compute; there is no other use.
+_LIB_PATH = Path(os.environ.get("CONCUR_ATTN_LIBRARY") or Path(__file__).resolve().parent / "libconcur_attn.so")
 
 CONCUR_OK = 0
 CONCUR_ERR_INVALID_ARG = -1
@@ -22,6 +26,7 @@ CONCUR_FLAG_BAD_PAGE_ID = 1
 CONCUR_FLAG_BAD_SEQ_LEN = 2
 CONCUR_FLAG_WAIT_LIMIT = 4
 CONCUR_FLAG_BAD_GROUP = 8
+CONCUR_FLAG_BOUNDS = 16
 
 CONCUR_KV_HEAD_MAJOR = 0
 CONCUR_KV_TOKEN_MAJOR = 1

@@ -10,6 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libconcur_attn.so"
+BOUNDS_LIB = PKG / "libconcur_attn_bounds.so"
 BENCH_CSRC = PKG / "bench_csrc"
 BENCH_LIB = PKG / "libconcur_bench.so"
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -35,9 +36,9 @@ def needs_build() -> bool:
     return any(d.stat().st_mtime > t for d in deps)
 
 
-def _compile(lib: Path, srcs, verbose: bool) -> None:
+def _compile(lib: Path, srcs, verbose: bool, defines=()) -> None:
     tmp = lib.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp), *map(str, srcs)]
+    cmd = [_nvcc(), *NVCC_FLAGS, *defines, *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp), *map(str, srcs)]
     subprocess.run(cmd, check=True)
     os.replace(tmp, lib)
 
@@ -51,6 +52,17 @@ def build_bench(force: bool = False, verbose: bool = False) -> Path:
     return BENCH_LIB
 
 
+def build_bounds(force: bool = False, verbose: bool = False) -> Path:
+    """The checked build: the same sources with -DCONCUR_BOUNDS, in which every index the kernels compute
+    for the workspace, the partial buffers and the outputs is held against its buffer's capacity
+    (a violation is recorded as CONCUR_FLAG_BOUNDS and the access skipped).  Load it by setting
+    CONCUR_ATTN_LIBRARY to its path before importing the package."""
+    deps = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list((PKG.parent / "include").glob("*.h"))
+    if force or not BOUNDS_LIB.exists() or any(d.stat().st_mtime > BOUNDS_LIB.stat().st_mtime for d in deps):
+        _compile(BOUNDS_LIB, sources(), verbose, ("-DCONCUR_BOUNDS",))
+    return BOUNDS_LIB
+
+
 def build(force: bool = False, verbose: bool = False) -> Path:
     build_bench(force, verbose)
     if not force and not needs_build():
@@ -61,4 +73,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
 
 if __name__ == "__main__":
     import sys
-    print(build(force=True, verbose="-v" in sys.argv))
+    if "--bounds" in sys.argv:
+        print(build_bounds(force=True, verbose="-v" in sys.argv))
+    else:
+        print(build(force=True, verbose="-v" in sys.argv))

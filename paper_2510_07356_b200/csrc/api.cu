@@ -176,6 +176,8 @@ static int fill_params(concur_attn_t* h, DecodeParams& p, const void* q, const v
     p.ranges_per_cta = h->ranges_per_cta;                 // 0: chosen per call from the amount of work
     p.min_range_tiles = h->min_range_tiles > 0 ? h->min_range_tiles : 2;
     p.max_ranges = kMaxRanges;
+    p.slot_cap = 2 * kMaxRanges;
+    p.out_rows = (int64_t)batch * h->cfg.num_q_heads;
     p.fuse_combine = h->fuse_combine;
     p.claim_ahead = h->claim_ahead;
     p.wait_limit_ns = h->wait_limit_ns;
@@ -391,6 +393,7 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
     c.prefix_lens = prefix_lens;
     c.num_groups = num_groups;
     c.grid_ctas = h->sm_count;
+    c.max_rows = lay.max_rows;
     c.chdr = reinterpret_cast<int32_t*>(cw + lay.chdr);
     c.tok_offset = reinterpret_cast<int32_t*>(cw + lay.tok_offset);
     c.seq_group = reinterpret_cast<int32_t*>(cw + lay.seq_group);
@@ -401,6 +404,7 @@ int concur_decode_attn_cascade(concur_attn_t* h, const void* q, const void* k_pa
     // the suffix pass writes one partial per segment into the cascade's own slots
     p.part_lse = reinterpret_cast<float*>(cw + lay.part_lse);
     p.part_o = reinterpret_cast<float*>(cw + lay.part_o);
+    p.slot_cap = lay.max_slots;
     p.tok_offset = c.tok_offset;
     p.all_partial = 1;
     p.fuse_combine = 0;
@@ -434,6 +438,7 @@ int concur_prefill_attn(concur_attn_t* h, const void* q, const void* k_pages, co
     fill_params(h, p, q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, batch, num_pages,
                 block_table_stride);
     p.grid_ctas = h->grid_ctas > 0 ? h->grid_ctas : h->sm_count;
+    p.out_rows = (int64_t)total_q * h->cfg.num_q_heads;
     PrefillParams f;
     f.q_start = q_start;
     f.total_q = total_q;

@@ -32,6 +32,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(
         const int64_t row = token_major ? ((int64_t)page * page_size + slot) * hkv + g
                                         : ((int64_t)page * hkv + g) * page_size + slot;
         const int64_t src = ((int64_t)b * hkv + g) * (kRowBytes / 16) + piece;
+        if (!in_bounds(hdr, row, (int64_t)num_pages * hkv * page_size, 601)) return;
         k_pages[row * (kRowBytes / 16) + piece] = k_new[src];
         v_pages[row * (kRowBytes / 16) + piece] = v_new[src];
     }

@@ -136,6 +136,25 @@ static_assert(TSmem<false>::kQOff % 1024 == 0 && TSmem<true>::kQOff % 1024 == 0 
               TCfg<false>::kQHalfBytes % 1024 == 0 && TCfg<true>::kQHalfBytes % 1024 == 0,
               "operand slabs must be 1024-byte aligned");
 static_assert(TSmem<false>::kBytes <= 232448 && TSmem<true>::kBytes <= 232448, "exceeds the 227 KB a CTA may use");
+// Extents of what the tensor-core descriptors read, against what the CTA owns.  (A 128-row operand read over
+// 80 staged rows once ran 1.6 KB past the CTA's allocation; this is the arithmetic that would have caught it.)
+//   Q.K^T, A operand: 128 rows x 128 B from the start of each half of a query buffer, the K = 16 steps up to 96 B
+//   further in: the last buffer's second half must still have 128 rows of the CTA's memory behind it.
+template <bool kPrefill>
+constexpr int q_read_end() {
+    return TSmem<kPrefill>::kQOff + TCfg<kPrefill>::kQBytes + TCfg<kPrefill>::kQHalfBytes + kTRows * 128;
+}
+static_assert(q_read_end<false>() <= TSmem<false>::kXchOff && q_read_end<true>() <= TSmem<true>::kXchOff,
+              "the 128-row query operand read must end inside the query buffers and their pad");
+//   Q.K^T, B operand: 64 token rows x 128 B per half of a K stage; P.V, B operand: per K = 16 step 16 token
+//   rows (2,048 B) of both halves of a V stage.
+static_assert(kTHalfBytes == kTile * 128 && 2 * kTHalfBytes == kTTileBytes && 4 * 2048 == kTHalfBytes,
+              "a K or V stage is two 64-row halves; four 16-token steps span a half");
+static_assert(TSmem<false>::kVOff == TCfg<false>::kKStages * kTTileBytes && TSmem<true>::kVOff == TCfg<true>::kKStages * kTTileBytes &&
+              TSmem<false>::kQOff == TSmem<false>::kVOff + TCfg<false>::kVStages * kTTileBytes &&
+              TSmem<true>::kQOff == TSmem<true>::kVOff + TCfg<true>::kVStages * kTTileBytes,
+              "K ring, V ring and query buffers follow one another without overlap");
+static_assert(64 + 64 + 64 + 32 + 32 + 128 + 128 == (int)kTmemCols, "three score buffers, two P tiles, two accumulators fill the 512 columns");
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, int32_t c2,
                                             uint32_t bar) {
@@ -633,7 +652,9 @@ attn_tc_kernel(DecodeParams p, CascadeParams c, PrefillParams f, const __grid_co
                     const float inv = 1.f / L;
                     const float f1 = w1 * inv, f2 = w2 * inv;
                     // prefix pass: a normalised fp32 partial per sibling; prefill: the final rows of out / lse
-                    const bool live = j < mt.n && (!kPrefill || head < p.group);
+                    const bool live = j < mt.n && (!kPrefill || head < p.group) &&
+                                      (kPrefill ? in_bounds(p.hdr, (int64_t)(mt.row + j) * p.hq + mt.g * p.group + head, p.out_rows, 201)
+                                                : in_bounds(p.hdr, mt.row + j, c.max_rows, 202));
                     float* dst = c.pre_o + ((int64_t)(mt.row + j) * kGroup + head) * kD + g * 64;
                     const int64_t out_row = (int64_t)(mt.row + j) * p.hq + mt.g * p.group + head;
                     #pragma unroll

@@ -30,6 +30,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(DecodeParams p
     // the unit's segment in range r is the range's first segment unless the range began
     // before the unit did (possible for r_lo only)
     const int32_t slot_lo = 2 * r_lo + (p.range_start[r_lo] < unit_start ? 1 : 0);
+    if (!in_bounds(p.hdr, slot_lo, p.slot_cap, 501) || !in_bounds(p.hdr, 2 * r_hi, p.slot_cap, 502) ||
+        !in_bounds(p.hdr, row0 + p.group - 1, p.out_rows, 503))
+        return;
     for (int h = 0; h < p.group; ++h) {
         float M = p.part_lse[(int64_t)slot_lo * kGroup + h];
         for (int32_t r = r_lo + 1; r <= r_hi; ++r)
@@ -87,6 +90,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(Decode
         const int32_t r_lo = range_of(W, R, unit_start), r_hi = range_of(W, R, unit_start + tiles_b - 1);
         for (int32_t r = r_lo; r <= r_hi; ++r) {
             const int64_t slot = (int64_t)r + b * p.hkv + g;
+            if (!in_bounds(p.hdr, slot, p.slot_cap, 504)) continue;
             add(p.part_lse + slot * kGroup, p.part_o + slot * kGroup * kD);
         }
     }
@@ -102,6 +106,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_cascade_kernel(Decode
         const int64_t row0 = c.unit_rowbase[i * p.hkv + g] + (b - b0);
         for (int32_t s = 0; s < splits; ++s) {
             const int64_t row = row0 + (int64_t)s * n;
+            if (!in_bounds(p.hdr, row, c.max_rows, 505)) continue;
             add(c.pre_lse + row * kGroup, c.pre_o + row * kGroup * kD);
         }
     }

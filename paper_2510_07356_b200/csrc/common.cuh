@@ -19,6 +19,7 @@ constexpr uint32_t kFlagBadPage = 1u;
 constexpr uint32_t kFlagBadLen = 2u;
 constexpr uint32_t kFlagWaitLimit = 4u;
 constexpr uint32_t kFlagBadGroup = 8u;
+constexpr uint32_t kFlagBounds = 16u;       // checked build only: an index the kernels computed fell outside its buffer
 
 // Workspace header (int32 words).
 enum HeaderWord : int {
@@ -29,6 +30,7 @@ enum HeaderWord : int {
     kHdrWaitSite = 4,     // which wait gave up first (diagnostic; 0 = none)
     kHdrClaimSelf = 5,    // launches without a plan kernel: ranges claimed so far beyond one per CTA; the
                           // launch's last claim puts it back to 0
+    kHdrBoundsSite = 7,   // checked build: which check failed first (diagnostic; 0 = none)
     kHdrWords = 64
 };
 
@@ -61,6 +63,9 @@ struct DecodeParams {
     int32_t ranges_per_cta;
     int32_t min_range_tiles;
     int32_t max_ranges;       // capacity of range_start / partial slots
+    // capacities, for the checked build (-DCONCUR_BOUNDS) to hold computed indices against
+    int32_t slot_cap;         // partial slots that part_o / part_lse hold
+    int64_t out_rows;         // rows ([Hq-indexed]) of out / lse
     int32_t fuse_combine;     // tensor-core kernel: 1 = the last partial of a unit merges it in-kernel
     int32_t claim_ahead;      // tiles before a range's end at which the next range is claimed
     int32_t no_plan_launch;   // tensor-core partial kernel: 1 = no plan kernel ran before this launch.  Ranges are
@@ -101,6 +106,7 @@ struct CascadeParams {
     int32_t* seq_group;           // [batch] group of each sequence
     int32_t* ptiles_prefix;       // [num_groups + 1] exclusive prefix of shared tiles per group
     int32_t* unit_rowbase;        // [num_groups * hkv + 1] first partial row of each prefix unit
+    int32_t max_rows;             // rows that pre_o / pre_lse hold (checked build)
     float* pre_o;                 // [rows][kGroup][kD] normalised partials of the prefix pass; rows = 8 x max batch
                                   // + 10 x CTAs: every unit's siblings once, plus once more per range cut
     float* pre_lse;               // [rows][kGroup]     their base-2 log-sum-exp
@@ -111,6 +117,21 @@ struct PrefillParams {
     const int32_t* q_start;       // [batch + 1] first query token of each sequence in q / out; last entry = total_q
     int32_t total_q;
 };
+
+// The checked build (-DCONCUR_BOUNDS) in place of a memory checker: every index a kernel computes for the
+// workspace, the partial buffers or the outputs is held against its buffer's capacity first; a violation is
+// recorded (CONCUR_FLAG_BOUNDS and the site of the first one) and the access is skipped instead of made.  In
+// the normal build the check is the constant `true` and costs nothing.
+#ifdef CONCUR_BOUNDS
+__device__ __forceinline__ bool in_bounds(int32_t* hdr, int64_t idx, int64_t cap, int site) {
+    if (idx >= 0 && idx < cap) return true;
+    atomicOr(reinterpret_cast<unsigned int*>(hdr + kHdrStatus), kFlagBounds);
+    atomicCAS(hdr + kHdrBoundsSite, 0, site);
+    return false;
+}
+#else
+__device__ __forceinline__ bool in_bounds(int32_t*, int64_t, int64_t, int) { return true; }
+#endif
 
 // Where token `slot` of KV head g of page `page` sits, as the (row, half-plane) coordinates of the
 // tensor maps over a pool (a row is 64 elements of one half of one 128-wide K or V row; `half` is

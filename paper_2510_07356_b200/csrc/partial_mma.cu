@@ -88,6 +88,17 @@ struct Smem {
 };
 constexpr int kSmemBytes = Smem::kTotal + 1024;           // slack for the manual 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may use");
+// What the copies write and the fragment loads read stays inside the tile it belongs to, for every box
+// size: a tile is 64 / P boxes of [2 halves][P rows][128 B]; the farthest byte a ldmatrix (or a lane copy,
+// or the fused append's patch) touches is the last 16-byte piece of the last row of the second half of the
+// last box.
+constexpr int tile_extent(int P) { return (kTile / P - 1) * P * kRowBytes + P * 128 + (P - 1) * 128 + 7 * 16 + 16; }
+static_assert(tile_extent(16) == kTileBytes && tile_extent(32) == kTileBytes && tile_extent(64) == kTileBytes,
+              "a tile's boxes must fill exactly its 16 KB");
+static_assert(2 * kTileBytes + kQBytes == kStageBytes && kGroup * kRowBytes == kQBytes, "stage = K tile | V tile | query rows");
+static_assert(Smem::kMergeOff == kStages * kStageBytes && Smem::kMlOff - Smem::kMergeOff == kMergeBytes &&
+              kMergeBytes >= kConsumerWarps * kGroup * kMergeStride * 4, "merge buffers follow the ring");
+static_assert((int)sizeof(StageMeta) % 16 == 0 && Smem::kBarOff % 8 == 0, "records and barriers are aligned");
 
 }  // namespace
 
@@ -468,6 +479,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
             if (lane == 0) mbar_arrive(job_taken);
             if (jexit) return;
             int32_t ticket = 0;
+            if (!in_bounds(p.hdr, jb * p.hkv + jg, (int64_t)p.batch * p.hkv, 101)) continue;
             if (lane == 0)
                 asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;"
                              : "=r"(ticket) : "l"(p.unit_done + jb * p.hkv + jg), "r"(1) : "memory");
@@ -489,6 +501,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
             #pragma unroll 2
             for (int32_t i = 0; i < splits; ++i) {
                 const int64_t slot = i ? 2 * (int64_t)(r_lo + i) : slot_lo;
+                if (!in_bounds(p.hdr, slot, p.slot_cap, 102)) continue;
                 const float4* lp = reinterpret_cast<const float4*>(p.part_lse + slot * kGroup);
                 const float4 la = __ldcg(lp), lb = __ldcg(lp + 1);
                 const float l8[kGroup] = {la.x, la.y, la.z, la.w, lb.x, lb.y, lb.z, lb.w};
@@ -511,6 +524,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                 if (h >= p.group) break;
                 const float inv = 1.f / z[h];
                 const int64_t row = (int64_t)jb * p.hq + jg * p.group + h;
+                if (!in_bounds(p.hdr, row, p.out_rows, 103)) continue;
                 uint2 packed;
                 packed.x = pack_bf16(acc[h].x * inv, acc[h].y * inv);
                 packed.y = pack_bf16(acc[h].z * inv, acc[h].w * inv);
@@ -607,7 +621,8 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                                  "r"(new_piece.y), "r"(new_piece.z), "r"(new_piece.w) : "memory");
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
-                if (mt.new_page >= 0) {
+                if (mt.new_page >= 0 && in_bounds(p.hdr, mt.new_page, p.num_pages, 106) &&
+                    in_bounds(p.hdr, mt.new_slot, p.page_size, 107) && in_bounds(p.hdr, patch_off, kTileBytes - 15, 108)) {
                     see_plan();
                     __nv_bfloat16* pool = lane < 16 ? const_cast<__nv_bfloat16*>(p.k_pages) : const_cast<__nv_bfloat16*>(p.v_pages);
                     *reinterpret_cast<uint4*>(pool + pool_elem(p, mt.new_page, mt.g, mt.new_slot) + (lane & 15) * 8) = new_piece;
@@ -745,14 +760,14 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                 hi.x *= inv; hi.y *= inv; hi.z *= inv; hi.w *= inv;
                 const float lse2 = M + log2f(L);
                 if (mt.slot < 0) {
-                    if (h < p.group) {
+                    if (h < p.group && in_bounds(p.hdr, (int64_t)mt.b * p.hq + mt.g * p.group + h, p.out_rows, 104)) {
                         const int64_t row = (int64_t)mt.b * p.hq + mt.g * p.group + h;
                         __nv_bfloat16* dst = p.out + row * kD + j4;
                         *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w));
                         *reinterpret_cast<uint2*>(dst + 64) = make_uint2(pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
                         if (j4 == 0) p.lse[row] = lse2 * 0.6931471805599453f;
                     }
-                } else {
+                } else if (in_bounds(p.hdr, mt.slot, p.slot_cap, 105)) {
                     const int64_t row = (int64_t)mt.slot * kGroup + h;
                     float* dst = p.part_o + row * kD + j4;
                     *reinterpret_cast<float4*>(dst) = lo;

@@ -177,12 +177,12 @@ __global__ void __launch_bounds__(kScalarThreads, 2) partial_scalar_kernel(Decod
                 const float res = acc / L;
                 const float lse2 = M + log2f(L);
                 if (sg.slot < 0) {
-                    if (h < p.group) {
+                    if (h < p.group && in_bounds(p.hdr, (int64_t)sg.b * p.hq + sg.g * p.group + h, p.out_rows, 401)) {
                         const int64_t row = (int64_t)sg.b * p.hq + sg.g * p.group + h;
                         p.out[row * kD + d] = __float2bfloat16_rn(res);
                         if (d == 0) p.lse[row] = lse2 * 0.6931471805599453f;
                     }
-                } else {
+                } else if (in_bounds(p.hdr, sg.slot, p.slot_cap, 402)) {
                     const int64_t row = (int64_t)sg.slot * kGroup + h;
                     p.part_o[row * kD + d] = res;
                     if (d == 0) p.part_lse[row] = lse2;

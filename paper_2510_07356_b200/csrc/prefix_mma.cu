@@ -387,6 +387,7 @@ prefix_mma_kernel(DecodeParams p, CascadeParams c, const __grid_constant__ CUten
                         L1 += lsum[(w * NS + j) * kGroup + 2 * quad + 1];
                     }
                     const float i0 = 1.f / L0, i1 = 1.f / L1;
+                    if (!in_bounds(p.hdr, mt.row + j, c.max_rows, 301)) continue;
                     float* dst = c.pre_o + ((int64_t)(mt.row + j) * kGroup) * kD;
                     #pragma unroll
                     for (int db = 0; db < 2; ++db) {

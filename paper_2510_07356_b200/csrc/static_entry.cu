@@ -119,6 +119,8 @@ extern "C" int concur_decode_attn_static(const void* q, const void* k_pages, con
     p.ranges_per_cta = 0;
     p.min_range_tiles = 2;
     p.max_ranges = kStaticMaxRanges;
+    p.slot_cap = 2 * kStaticMaxRanges;
+    p.out_rows = (int64_t)batch * kHq;
     p.fuse_combine = 1;
     p.claim_ahead = 1 << 20;
     p.wait_limit_ns = 2000000000ll;
