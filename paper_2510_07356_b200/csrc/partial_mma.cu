@@ -62,7 +62,7 @@ struct StageMeta {
     int32_t new_row;       // fused append: row of the tile that is the sequence's new token, else -1
     int32_t new_page;      // ... and the pool page its slot is in (-1: not to be stored, the page id was bad)
     int32_t seg_new;       // fused append: 1 on a segment's first tile if the segment holds the unit's last tile
-    int32_t new_slot;      // fused append: slot of the new token inside new_page
+    int32_t row_in_page;   // first row of the tile inside its page (non-zero only for pages of more than 64 tokens)
 };
 
 // A finished partial segment handed from the consumer warps to the combiner warp.
@@ -273,8 +273,54 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
     };
 
     if (warp >= kCopyWarp0) {
-        // =========================================================== copy helper warps (small pages)
-        if (!lane_copy) return;
+        // =========================================================== helper warps
+        if (!lane_copy) {
+            // Pages of 64 tokens or more: the producer only keeps the books (ranges, segments, page ids, the
+            // tile's record); the first helper issues the K copy (and a segment's query rows) of every tile
+            // from that record, the second one the V copy.  Arming a barrier and issuing a tensor copy are
+            // slow serial steps of one thread; with all of them in the producer its time per tile, not HBM,
+            // set the kernel's rate (the step time times the SM clock was a constant).
+            if (warp > kCopyWarp0 + 1) return;
+            const bool is_k = warp == kCopyWarp0;
+            const uint32_t box_bytes = (uint32_t)P * kRowBytes;
+            uint32_t it = 0;
+            bool ok = true;
+            for (;; ++it) {
+                const int s = it % kStages;
+                ok = mbar_wait(sched(s), (it / kStages) & 1u, abort_flag, wait_ns);
+                if (!ok) break;
+                const int32_t n_valid = meta[s].n_valid;
+                if (n_valid == 0) return;
+                if (lane == 0) {
+                    const int32_t npages = (n_valid + P - 1) >> p.box_shift;
+                    const int32_t g = meta[s].g, rip = meta[s].row_in_page;
+                    const uint32_t kdst = smem_base + s * kStageBytes;
+                    if (is_k) {
+                        const bool with_q = meta[s].first != 0;
+                        const uint32_t q_bytes = (uint32_t)p.group * kRowBytes;
+                        mbar_arrive_expect_tx(full_k(s), npages * box_bytes + (with_q ? q_bytes : 0u));
+                        if (with_q)
+                            bulk_load(kdst + 2 * kTileBytes, p.q + ((int64_t)meta[s].b * p.hq + g * p.group) * kD, q_bytes, full_k(s));
+                        for (int i = 0; i < npages; ++i)
+                            tma_load_tile(kdst + i * box_bytes, &map_k, pool_row(p, meta[s].page[i], g, rip), full_k(s), pool_plane(p, g));
+                    } else {
+                        mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
+                        for (int i = 0; i < npages; ++i)
+                            tma_load_tile(kdst + kTileBytes + i * box_bytes, &map_v, pool_row(p, meta[s].page[i], g, rip), full_v(s), pool_plane(p, g));
+                    }
+                }
+                __syncwarp();
+            }
+            // a wait gave up (here or elsewhere in the CTA): let this warp's copies in flight land before
+            // the CTA's shared memory is released
+            if (lane == 0) {
+                wait_failed(p, abort_flag, 11);
+                volatile int32_t never = 0;
+                for (uint32_t j = it > (uint32_t)kStages ? it - kStages : 0u; j < it; ++j)
+                    mbar_wait(is_k ? full_k(j % kStages) : full_v(j % kStages), (j / kStages) & 1u, &never);
+            }
+            return;
+        }
         const int w = warp - kCopyWarp0 + 1;
         for (uint32_t it = 0;; ++it) {
             const int s = it % kStages;
@@ -293,7 +339,6 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
         uint32_t it = 0;                       // tiles issued so far
         int32_t r = blockIdx.x;                // CTA i starts on range i; further ranges are claimed
         bool ok = true;
-        const uint32_t box_bytes = (uint32_t)P * kRowBytes;
         const int32_t page_mask = p.page_size - 1;
         while (ok && r < R) {
             // the next range is claimed a few tiles before this one ends: late enough that no
@@ -365,35 +410,25 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                             // fused append: the sequence's last token sits in the unit's last tile
                             const bool new_here = p.k_new != nullptr && t == sg.tiles_b - 1;
                             const int32_t new_row = n_valid - 1;
-                            const int32_t new_pages[4] = {page0, page1, page2, page3};
+                            const int32_t new_box = new_row >> p.box_shift;
+                            const int32_t new_page = new_box == 0 ? page0 : (new_box == 1 ? page1 : (new_box == 2 ? page2 : page3));
                             m.new_row = new_here ? new_row : -1;
-                            m.new_page = (new_here && !new_page_bad) ? new_pages[new_row >> p.box_shift] : -1;
+                            m.new_page = (new_here && !new_page_bad) ? new_page : -1;
                             m.seg_new = (p.k_new != nullptr && sg.tile1 == sg.tiles_b) ? 1 : 0;
-                            m.new_slot = (tok_abs + new_row) & page_mask;
-                            const uint32_t kdst = smem_base + s * kStageBytes;
-                            const uint32_t vdst = kdst + kTileBytes;
-                            const bool with_q = (t == sg.tile0);
-                            const uint32_t q_bytes = (uint32_t)p.group * kRowBytes;
-                            const uint32_t tile_tx = lane_copy ? 0u : npages * box_bytes;
-                            const uint32_t tx = tile_tx + (with_q ? q_bytes : 0);
-                            if (tx) mbar_arrive_expect_tx(full_k(s), tx);
-                            else mbar_arrive(full_k(s));
-                            if (with_q)
-                                bulk_load(vdst + kTileBytes, p.q + ((int64_t)sg.b * p.hq + sg.g * p.group) * kD,
-                                          q_bytes, full_k(s));
-                            if (lane_copy) mbar_arrive(sched(s));          // the helpers may read the record
-                            if (!lane_copy) {
-                                const int32_t pages[4] = {page0, page1, page2, page3};
-                                #pragma unroll
-                                for (int i = 0; i < 4; ++i)
-                                    if (i < npages)
-                                        tma_load_tile(kdst + i * box_bytes, &map_k, pool_row(p, pages[i], sg.g, row_in_page), full_k(s), pool_plane(p, sg.g));
-                                mbar_arrive_expect_tx(full_v(s), npages * box_bytes);
-                                #pragma unroll
-                                for (int i = 0; i < 4; ++i)
-                                    if (i < npages)
-                                        tma_load_tile(vdst + i * box_bytes, &map_v, pool_row(p, pages[i], sg.g, row_in_page), full_v(s), pool_plane(p, sg.g));
+                            m.row_in_page = row_in_page;
+                            if (lane_copy) {
+                                // small pages: the query rows by a bulk copy from here; the tile itself by the
+                                // per-lane copies of this warp and the three helpers
+                                const uint32_t kdst = smem_base + s * kStageBytes;
+                                const bool with_q = (t == sg.tile0);
+                                const uint32_t q_bytes = (uint32_t)p.group * kRowBytes;
+                                if (with_q) mbar_arrive_expect_tx(full_k(s), q_bytes);
+                                else mbar_arrive(full_k(s));
+                                if (with_q)
+                                    bulk_load(kdst + 2 * kTileBytes, p.q + ((int64_t)sg.b * p.hq + sg.g * p.group) * kD,
+                                              q_bytes, full_k(s));
                             }
+                            mbar_arrive(sched(s));          // the helper warps may read the record (and issue the copies)
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -420,14 +455,15 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                 if (ok) {
                     meta[s].n_valid = 0;
                     mbar_arrive_n(full_k(s), lane_copy ? 1 + kCopyLanes : 1);
-                    if (lane_copy) mbar_arrive(sched(s));
+                    mbar_arrive(sched(s));
                 }
             }
             if (!ok) {
                 wait_failed(p, abort_flag, 1);
-                // let the copies still in flight land before the CTA's shared memory is released
+                // let the copies still in flight land before the CTA's shared memory is released (small pages:
+                // this warp's own; otherwise the helper warps issued them and wait for them)
                 const uint32_t lo = it > (uint32_t)kStages ? it - kStages : 0u;
-                for (uint32_t j = lo; j < it; ++j) {
+                for (uint32_t j = lane_copy ? lo : it; j < it; ++j) {
                     volatile int32_t never = 0;
                     mbar_wait(full_k(j % kStages), (j / kStages) & 1u, &never);
                     mbar_wait(full_v(j % kStages), (j / kStages) & 1u, &never);
@@ -606,28 +642,34 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                     (lane < 16 ? p.k_new : p.v_new) + ((int64_t)mt.b * p.hkv + mt.g) * kD + (lane & 15) * 8));
         }
         const int valid = mt.n_valid - tok0;          // valid tokens among this warp's 16
-        // fused append: is the new token one of this warp's rows of this tile?
-        const bool patch = mt.new_row >= tok0 && mt.new_row < tok0 + 16;
-        // where the 16-byte piece (lane & 15) of that row sits in a swizzled tile (relative to the tile's base)
-        const uint32_t patch_off = (uint32_t)(mt.new_row >> p.box_shift) * (uint32_t)P * kRowBytes +
-                                   (uint32_t)((lane & 15) >> 3) * half_stride + (uint32_t)(mt.new_row & (P - 1)) * 128u +
-                                   (uint32_t)((((lane & 15) & 7) ^ (mt.new_row & 7)) << 4);
-        if (valid > 0) {
+        // Fused append (one tile per unit, none in any other call): the tile holds the sequence's new token.
+        // The pool's slot has not been written yet, so the warp that owns the row puts the K row (here) and the
+        // V row (below, once V has landed) where the copy left the slot's old contents, and stores both rows
+        // into the pools for the steps to come.  patch_off: where the 16-byte piece (lane & 15) of the row sits
+        // in a swizzled tile.
+        bool patch = false;
+        uint32_t patch_off = 0;
+        if (mt.new_row >= 0) {
+            patch = mt.new_row >= tok0 && mt.new_row < tok0 + 16;
+            patch_off = (uint32_t)(mt.new_row >> p.box_shift) * (uint32_t)P * kRowBytes +
+                        (uint32_t)((lane & 15) >> 3) * half_stride + (uint32_t)(mt.new_row & (P - 1)) * 128u +
+                        (uint32_t)((((lane & 15) & 7) ^ (mt.new_row & 7)) << 4);
             if (patch) {
-                // the pool's slot has not been written yet: put the K row where the copy left the slot's old
-                // contents, and store both rows into the pools for the steps to come
                 if (lane < 16)
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(kbase + patch_off), "r"(new_piece.x),
                                  "r"(new_piece.y), "r"(new_piece.z), "r"(new_piece.w) : "memory");
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (mt.new_page >= 0 && in_bounds(p.hdr, mt.new_page, p.num_pages, 106) &&
-                    in_bounds(p.hdr, mt.new_slot, p.page_size, 107) && in_bounds(p.hdr, patch_off, kTileBytes - 15, 108)) {
+                    in_bounds(p.hdr, patch_off, kTileBytes - 15, 108)) {
                     see_plan();
+                    const int32_t new_slot = (mt.row_in_page + mt.new_row) & (p.page_size - 1);
                     __nv_bfloat16* pool = lane < 16 ? const_cast<__nv_bfloat16*>(p.k_pages) : const_cast<__nv_bfloat16*>(p.v_pages);
-                    *reinterpret_cast<uint4*>(pool + pool_elem(p, mt.new_page, mt.g, mt.new_slot) + (lane & 15) * 8) = new_piece;
+                    *reinterpret_cast<uint4*>(pool + pool_elem(p, mt.new_page, mt.g, new_slot) + (lane & 15) * 8) = new_piece;
                 }
             }
+        }
+        if (valid > 0) {
             // ---- S^T = K . Q^T  (two accumulator chains to shorten the dependency)
             float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
             #pragma unroll
