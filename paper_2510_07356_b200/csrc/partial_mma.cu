@@ -1,9 +1,9 @@
 // Split-KV partial kernel, tensor-core version (the default).
 //
-// One persistent CTA per SM: a producer warp streams K and V tiles (64 tokens x 128 dims,
-// 16 KB each) from the paged pools into a 6-stage shared-memory ring with TMA tensor
-// copies (128-byte swizzle, one copy per (page, KV head) chunk), four consumer warps
-// each own 16 tokens of every tile:
+// One persistent CTA per SM: K and V tiles (64 tokens x 128 dims, 16 KB each) are streamed from the
+// paged pools into a 5-stage shared-memory ring with TMA tensor copies (128-byte swizzle, one copy
+// per (page, KV head) chunk).  Two sets of four consumer warps take alternate tiles; within a set
+// each warp owns 16 tokens of the tile:
 //
 //   S^T[16 tok x 8 heads]  = K[16 tok x 128] . Q^T[128 x 8]        (8 mma.m16n8k16, bf16 -> fp32)
 //   online softmax in fp32, base-2 domain, per-warp running max / sum
@@ -38,11 +38,12 @@ namespace concur {
 
 namespace {
 
-constexpr int kStages = 6;
-constexpr int kConsumerWarps = 4;
-constexpr int kProducerWarp = kConsumerWarps;          // warp 4
-constexpr int kCombinerWarp = kConsumerWarps + 1;      // warp 5
-constexpr int kCopyWarp0 = kConsumerWarps + 2;         // warps 6-8: copy helpers, used with small pages only
+constexpr int kStages = 5;
+constexpr int kSetWarps = 4;                           // warps of a consumer set: 16 tokens of a tile each
+constexpr int kConsumerWarps = 2 * kSetWarps;          // set 0 (warps 0-3) takes even tiles, set 1 (warps 4-7) odd ones
+constexpr int kProducerWarp = kConsumerWarps;          // warp 8
+constexpr int kCombinerWarp = kConsumerWarps + 1;      // warp 9
+constexpr int kCopyWarp0 = kConsumerWarps + 2;         // warps 10-12: helpers (copy issue; per-lane copies with small pages)
 constexpr int kCopyWarps = 3;
 constexpr int kThreads = (kConsumerWarps + 2 + kCopyWarps) * 32;
 constexpr int kTileBytes = kTile * kRowBytes;             // 16 KB: one K or V tile
@@ -76,7 +77,7 @@ struct CombineJob {
 struct Smem {
     // offsets from the 1024-aligned base
     static constexpr int kMergeOff = kStages * kStageBytes;
-    static constexpr int kMlOff = kMergeOff + kMergeBytes;                       // [4 warps][8 heads][2]
+    static constexpr int kMlOff = kMergeOff + kMergeBytes;                       // [8 warps][8 heads][2]
     static constexpr int kPrefixOff = kMlOff + kConsumerWarps * kGroup * 2 * 4;  // [kSmemBatch + 1]
     static constexpr int kLenOff = kPrefixOff + (kSmemBatch + 1) * 4;            // [kSmemBatch + 1]
     static constexpr int kMetaOff = kLenOff + (kSmemBatch + 1) * 4;
@@ -141,7 +142,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
             mbar_init(full_k(s), lane_copy ? 1 + kCopyLanes : 1);
             mbar_init(full_v(s), lane_copy ? kCopyLanes : 1);
             mbar_init(sched(s), 1);
-            mbar_init(empty(s), kConsumerWarps);
+            mbar_init(empty(s), kConsumerWarps);       // the owning set when it is done, the other one when it has the record
         }
         mbar_init(merge_bar0, kConsumerWarps * 32);
         mbar_init(merge_bar1, kConsumerWarps * 32);
@@ -577,7 +578,11 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
     // per-lane pieces of the swizzled tile addresses (see the layout note at tma_load_tile):
     // a 64-token tile is 64/P boxes; a box is [2 halves][P rows][128 B], 16-byte chunks of a
     // row XOR-ed with (row & 7)
-    const int tok0 = warp * 16;                                   // this warp's first token in the tile
+    // Two sets: a warp's work on a tile is one dependent chain (fragment loads, 8 MMAs, shuffles, exponentials,
+    // transposes, 8 MMAs) with nothing of its own to overlap it with; two sets, each with its own running
+    // state, halve the time the consumer side needs per tile.
+    const int set = warp / kSetWarps;                             // this warp's set: tiles with (it & 1) == set
+    const int tok0 = (warp % kSetWarps) * 16;                     // this warp's first token in the tile
     const uint32_t box_off = (uint32_t)(tok0 >> p.box_shift) * (uint32_t)P * kRowBytes;
     const uint32_t half_stride = (uint32_t)P * 128u;
     const int rb0 = tok0 & (P - 1);
@@ -624,6 +629,10 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
         }
         const uint32_t kbase = smem_base + s * kStageBytes;
         const uint32_t vbase = kbase + kTileBytes;
+        // Both sets walk every tile's record: the segment's first tile carries its query rows (the set
+        // that does not own that tile needs them for the next one) and starts both sets' states afresh,
+        // and its last tile is where both meet for the merge.
+        const bool mine = (int)(it & 1u) == set;
         if (mt.first) {
             const uint32_t* qs = reinterpret_cast<const uint32_t*>(smem + s * kStageBytes + 2 * kTileBytes);
             #pragma unroll
@@ -641,7 +650,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                 new_piece = __ldg(reinterpret_cast<const uint4*>(
                     (lane < 16 ? p.k_new : p.v_new) + ((int64_t)mt.b * p.hkv + mt.g) * kD + (lane & 15) * 8));
         }
-        const int valid = mt.n_valid - tok0;          // valid tokens among this warp's 16
+        const int valid = mine ? mt.n_valid - tok0 : 0;          // valid tokens among this warp's 16
         // Fused append (one tile per unit, none in any other call): the tile holds the sequence's new token.
         // The pool's slot has not been written yet, so the warp that owns the row puts the K row (here) and the
         // V row (below, once V has landed) where the copy left the slot's old contents, and stores both rows
@@ -649,7 +658,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
         // in a swizzled tile.
         bool patch = false;
         uint32_t patch_off = 0;
-        if (mt.new_row >= 0) {
+        if (mt.new_row >= 0 && mine) {
             patch = mt.new_row >= tok0 && mt.new_row < tok0 + 16;
             patch_off = (uint32_t)(mt.new_row >> p.box_shift) * (uint32_t)P * kRowBytes +
                         (uint32_t)((lane & 15) >> 3) * half_stride + (uint32_t)(mt.new_row & (P - 1)) * 128u +
@@ -748,7 +757,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
         if (lane == 0) mbar_arrive(empty(s));
 
         if (mt.last) {
-            // ---- merge the four warps' states and write the segment's result
+            // ---- merge the eight warps' states (both sets) and write the segment's result
             see_plan();
             #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {
@@ -773,11 +782,12 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                 if (lane == 0) wait_failed(p, abort_flag, 4);
                 return;
             }
-            // 128 consumer threads = 8 heads x 16 threads; a thread owns dims 4j .. 4j+3 and 64+4j .. 64+4j+3
-            // of one head (16-byte pieces: conflict-free shared-memory reads, 8- or 16-byte stores), so
-            // the head's weights are computed once per thread instead of once per (thread, head)
+            // 256 consumer threads = 8 heads x 32 threads; a thread owns dims 4j .. 4j+3 of one head (a warp
+            // reads 512 contiguous bytes of every state: conflict-free; 8- or 16-byte stores), so the
+            // head's weights are computed once per thread instead of once per (thread, head).  A set
+            // that took no tile of the segment contributes m = -inf, l = 0, O = 0: weight 0.
             {
-                const int h = tid >> 4, j4 = (tid & 15) * 4;
+                const int h = tid >> 5, j4 = (tid & 31) * 4;
                 float2 ml[kConsumerWarps];
                 float M = ninf;
                 #pragma unroll
@@ -786,34 +796,28 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                     M = fmaxf(M, ml[w].x);
                 }
                 float L = 0.f;
-                float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) {
                     const float wt = fast_exp2(ml[w].x - M);
                     L = fmaf(ml[w].y, wt, L);
-                    const float* src = merge_o + (w * kGroup + h) * kMergeStride + j4;
-                    const float4 a = *reinterpret_cast<const float4*>(src);
-                    const float4 c = *reinterpret_cast<const float4*>(src + 64);
-                    lo.x = fmaf(a.x, wt, lo.x); lo.y = fmaf(a.y, wt, lo.y); lo.z = fmaf(a.z, wt, lo.z); lo.w = fmaf(a.w, wt, lo.w);
-                    hi.x = fmaf(c.x, wt, hi.x); hi.y = fmaf(c.y, wt, hi.y); hi.z = fmaf(c.z, wt, hi.z); hi.w = fmaf(c.w, wt, hi.w);
+                    const float4 a = *reinterpret_cast<const float4*>(merge_o + (w * kGroup + h) * kMergeStride + j4);
+                    acc.x = fmaf(a.x, wt, acc.x); acc.y = fmaf(a.y, wt, acc.y);
+                    acc.z = fmaf(a.z, wt, acc.z); acc.w = fmaf(a.w, wt, acc.w);
                 }
                 const float inv = 1.f / L;
-                lo.x *= inv; lo.y *= inv; lo.z *= inv; lo.w *= inv;
-                hi.x *= inv; hi.y *= inv; hi.z *= inv; hi.w *= inv;
+                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
                 const float lse2 = M + log2f(L);
                 if (mt.slot < 0) {
                     if (h < p.group && in_bounds(p.hdr, (int64_t)mt.b * p.hq + mt.g * p.group + h, p.out_rows, 104)) {
                         const int64_t row = (int64_t)mt.b * p.hq + mt.g * p.group + h;
-                        __nv_bfloat16* dst = p.out + row * kD + j4;
-                        *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w));
-                        *reinterpret_cast<uint2*>(dst + 64) = make_uint2(pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
+                        *reinterpret_cast<uint2*>(p.out + row * kD + j4) =
+                            make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
                         if (j4 == 0) p.lse[row] = lse2 * 0.6931471805599453f;
                     }
                 } else if (in_bounds(p.hdr, mt.slot, p.slot_cap, 105)) {
                     const int64_t row = (int64_t)mt.slot * kGroup + h;
-                    float* dst = p.part_o + row * kD + j4;
-                    *reinterpret_cast<float4*>(dst) = lo;
-                    *reinterpret_cast<float4*>(dst + 64) = hi;
+                    *reinterpret_cast<float4*>(p.part_o + row * kD + j4) = acc;
                     if (j4 == 0) p.part_lse[row] = lse2;
                 }
             }
