@@ -43,8 +43,8 @@ constexpr int kSetWarps = 4;                           // warps of a consumer se
 constexpr int kConsumerWarps = 2 * kSetWarps;          // set 0 (warps 0-3) takes even tiles, set 1 (warps 4-7) odd ones
 constexpr int kProducerWarp = kConsumerWarps;          // warp 8
 constexpr int kCombinerWarp = kConsumerWarps + 1;      // warp 9
-constexpr int kCopyWarp0 = kConsumerWarps + 2;         // warps 10-12: helpers (copy issue; per-lane copies with small pages)
-constexpr int kCopyWarps = 3;
+constexpr int kCopyWarp0 = kConsumerWarps + 2;         // warps 10-13: helpers (copy issue; per-lane copies with small pages)
+constexpr int kCopyWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 2 + kCopyWarps) * 32;
 constexpr int kTileBytes = kTile * kRowBytes;             // 16 KB: one K or V tile
 constexpr int kQBytes = kGroup * kRowBytes;               // 2 KB: the 8 query rows of a group
@@ -129,13 +129,15 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
     const int64_t max_len = (int64_t)p.bt_stride * p.page_size;
     const bool cached = p.batch <= kSmemBatch;
     // Small pages (16 or 32 tokens): a tile would be four or two TMA boxes per operand, and the copy
-    // engine's cost per box caps the stream well below HBM speed.  There the producer warp and three
-    // helper warps copy a quarter of the tile each (16 rows), 16 bytes per lane and instruction, into
-    // the same swizzled layout; a tile's barrier then takes one arrival per copying lane (when that
-    // lane's copies have landed) next to the producer's own.
+    // engine's cost per box caps the stream well below HBM speed.  There four helper warps copy a
+    // quarter of the tile each (16 rows), 16 bytes per lane and instruction, into the same swizzled
+    // layout; a tile's barrier then takes one arrival per copying lane (when that lane's copies have
+    // landed) next to the producer's own.  (The producer used to copy one of the quarters itself; as
+    // its time per tile is what the rate hangs on, giving that quarter to a fourth helper took 14 % off
+    // a step with 16-token pages.)
     const bool lane_copy = p.lane_copy != 0;
     const uint64_t wait_ns = (uint64_t)p.wait_limit_ns;       // the roles' waits; the drain of copies in flight keeps 2 s
-    constexpr uint32_t kCopyLanes = (1 + kCopyWarps) * 32;
+    constexpr uint32_t kCopyLanes = kCopyWarps * 32;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -322,7 +324,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
             }
             return;
         }
-        const int w = warp - kCopyWarp0 + 1;
+        const int w = warp - kCopyWarp0;
         for (uint32_t it = 0;; ++it) {
             const int s = it % kStages;
             if (!mbar_wait(sched(s), (it / kStages) & 1u, abort_flag, wait_ns)) {
@@ -419,7 +421,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                             m.row_in_page = row_in_page;
                             if (lane_copy) {
                                 // small pages: the query rows by a bulk copy from here; the tile itself by the
-                                // per-lane copies of this warp and the three helpers
+                                // per-lane copies of the four helper warps
                                 const uint32_t kdst = smem_base + s * kStageBytes;
                                 const bool with_q = (t == sg.tile0);
                                 const uint32_t q_bytes = (uint32_t)p.group * kRowBytes;
@@ -433,7 +435,6 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (ok && lane_copy) copy_quarter(s, 0, n_valid, sg.g, page0);
                     if (ok) ++it;
                 }
             }
