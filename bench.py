@@ -50,12 +50,12 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one partial_mma_kernel launch divided by its KV tokens, from
 # an ncu capture of a quarter of the 64 x 16,384 configuration (page size 64, fused combine, one range per
 # CTA).  Set to None whenever that kernel changes until the counters are taken again.
-MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074885e9 + 4.496384e6) / 262144
+MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074892e9 + 4.929280e6) / 262144
 # The same two counters of one attn_tc_kernel launch on exactly these workloads; None for any other
 # workload, and to be removed whenever that kernel changes until the counters are taken again.
 ATTN_TC_TRAFFIC_BYTES = {
-    ("casc_16x10_pre16384_p64", "tcgen05"): 1.080627e9 + 10.573312e6,
-    ("prefill_16x2048_p64", "tcgen05"): 671.279872e6 + 505.919488e6,
+    ("casc_16x10_pre16384_p64", "tcgen05"): 1.078966e9 + 10.120704e6,
+    ("prefill_16x2048_p64", "tcgen05"): 671.184640e6 + 506.286592e6,
 }
 
 
