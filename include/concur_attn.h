@@ -13,7 +13,7 @@
  * This is the attention step of the batched autoregressive decoding of long reasoning
  * traces on which the ConCuR pipeline (arXiv 2510.07356) spends its generation time:
  * five samples for each of 18,162 tasks by a 32B GQA model (Sec. 3.3), ten per task in
- * evaluation (Sec. 4.1), traces of 4,000-8,500 tokens and more (Tables 3 and 4) under a
+ * evaluation (Sec. 4.2), traces of 4,000-8,500 tokens and more (Tables 3 and 4) under a
  * 32,768-token limit (Sec. 4.1).  The paper states no formula for it; the definition
  * above is the standard one.
  *
@@ -223,7 +223,7 @@ int concur_decode_attn_planned(concur_attn_t* handle,
 /*
  * The same step when sequences share a cached prefix (cascade decode).  In the paper's
  * workload every task is sampled 5 times for synthesis and 10 times for evaluation from one
- * fixed prompt (Sec. 3.3, Sec. 4.1, App. C), so the samples of a task have their whole
+ * fixed prompt (Sec. 3.3, Sec. 4.2, App. C), so the samples of a task have their whole
  * prompt in common; with a paged cache they can point at the same physical pages.
  *
  *   group_start   device, int32 [num_groups + 1]: group i is sequences group_start[i] ..
@@ -260,7 +260,7 @@ int concur_decode_attn_cascade(concur_attn_t* handle,
  * Prefill: causal attention of several new query tokens per sequence against the cache -- the
  * step that runs once per prompt before its samples are decoded (in the paper's pipeline every
  * task's prompt, the fixed template of App. C around the task's program, is processed once and
- * then sampled 5 or 10 times, Sec. 3.3 / 4.1), or once per chunk of a long prompt.  The paper
+ * then sampled 5 or 10 times, Sec. 3.3 / 4.2), or once per chunk of a long prompt.  The paper
  * states no formula; per query token the definition is that of the decode step:
  *
  *   sequence b has q_len = q_start[b+1] - q_start[b] query tokens, rows q_start[b] .. of q, out
@@ -292,7 +292,7 @@ int concur_prefill_attn(concur_attn_t* handle,
  * for every sequence b, the new token's rows k_new[b][g][:], v_new[b][g][:] (g = 0..Hkv-1)
  * are stored at position pos = seq_lens[b], i.e. slot pos % P of page
  * block_table[b][pos / P], and seq_lens[b] becomes pos + 1.  (The generation loop whose
- * attention step this library implements -- Sec. 3.3 / 4.1 of the paper -- appends one
+ * attention step this library implements -- Sec. 3.3 / 4.2 of the paper -- appends one
  * token per sequence per step; the paper does not describe the cache.)
  *
  *   k_new, v_new   device, bf16 [batch][Hkv][D], 16-byte aligned

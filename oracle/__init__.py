@@ -6,7 +6,7 @@ path and imports nothing from it.  Only tests, the smoke check and the benchmark
 CPU-baseline leg may use it; the product path never does.
 
 Operation (the paper, arXiv 2510.07356, decodes long reasoning traces with 32B GQA
-models in Sec. 3.3 / Sec. 4.1 but states no formula; this is the textbook
+models in Sec. 3.3 / Sec. 4.2 but states no formula; this is the textbook
 definition): ``out = softmax(scale * q K^T) V`` per query head over the tokens a
 block table maps into a paged pool, ``lse = ln sum exp(scale * q k_j)``.
 
