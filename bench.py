@@ -10,7 +10,10 @@ WORLD_SIZE it is one of the ranks.  Either way the world size must equal N or th
 --shard replicas (default): every rank decodes its own batch of the workload's shape (weak scaling);
 --shard kv-heads: the ranks split ONE batch the way tensor parallelism does, each holding Hkv / N KV
 heads of every page and the query heads that attend to them (strong scaling, no collective inside
-attention).  NCCL carries only the barrier and the max / sum of the timings.
+attention); --shard context: every sequence's tokens are split by range, each rank attends to its range
+and the ranks' (out, lse) pairs are all-gathered (NCCL, 260 bytes per query row and rank) and merged by
+concur_lse_merge inside the timed step (strong scaling; the one exchange step this path can have).
+Otherwise NCCL carries only the barrier and the max / sum of the timings.
 
 NAME is one of synth.SPECS (plain decode step; the default is the 64 x 16,384 configuration) or of
 synth.CASCADE_SPECS (shared-prefix step: `value` counts the shared pages once, `logical_gbs` as if
@@ -66,8 +69,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
-    ap.add_argument("--shard", default="replicas", choices=["replicas", "kv-heads"],
-                    help="N > 1: independent batches per rank, or one batch split over the KV heads")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "kv-heads", "context"],
+                    help="N > 1: independent batches per rank, one batch split over the KV heads, or one batch "
+                         "split over every sequence's token range (partials gathered and merged)")
     ap.add_argument("--kernel", type=int, default=0, help="0 tensor-core partial kernel, 1 scalar-FMA")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -285,6 +289,8 @@ def rank_workload(spec, rank: int, world: int, shard: str, device, **kw):
         if spec.num_kv_heads % world:
             raise SystemExit(f"--shard kv-heads: {spec.num_kv_heads} KV heads do not split over {world} ranks")
         return synth.shard_kv_heads(synth.make_workload(spec, device, **kw), rank, world)
+    if shard == "context":
+        return synth.shard_context(synth.make_workload(spec, device, **kw), rank, world)
     return synth.make_workload(rank_spec(spec, rank, world), device, **kw)
 
 
@@ -898,6 +904,8 @@ def main():
         return
     if args.shard == "kv-heads" and args.workload.startswith(("casc", "prefill", "curate", "loop")):
         raise SystemExit("bench.py: --shard kv-heads is implemented for the plain decode workloads")
+    if args.shard == "context" and args.workload.startswith(("casc", "prefill", "curate", "loop")):
+        raise SystemExit("bench.py: --shard context is implemented for the plain decode workloads")
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # no outside launcher: this process becomes the launcher of its own N ranks
         raise SystemExit(spawn_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
@@ -951,8 +959,28 @@ def main():
     flush_needed = kv_bytes < 512 * 1024 * 1024          # inputs not well above the 126 MB L2
     flush_buf = L2Flush(dev) if flush_needed else None
 
+    ctx = args.shard == "context"
+    if ctx:
+        # every rank's (out, lse) over its token range, gathered from all ranks, then merged on every rank
+        args.loop_steps = 0
+        args.no_e2e = True
+        rows = spec.batch * spec.num_q_heads
+        out_part = torch.empty_like(w.q)
+        lse_part = torch.empty((spec.batch, spec.num_q_heads), dtype=torch.float32, device=dev)
+        gath_out = torch.empty((world,) + tuple(w.q.shape), dtype=torch.bfloat16, device=dev)
+        gath_lse = torch.empty((world, spec.batch, spec.num_q_heads), dtype=torch.float32, device=dev)
+
     def step():
-        attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale, out=out, lse=lse)
+        if not ctx:
+            attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale, out=out, lse=lse)
+            return
+        attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale, out=out_part, lse=lse_part)
+        if world > 1:
+            dist.all_gather_into_tensor(gath_out, out_part)
+            dist.all_gather_into_tensor(gath_lse, lse_part)
+        else:
+            gath_out[0].copy_(out_part); gath_lse[0].copy_(lse_part)
+        P.concur_lse_merge(gath_out, gath_lse, world, rows, out, lse, torch.cuda.current_stream(dev).cuda_stream)
 
     def barrier():
         if world > 1:
@@ -1181,14 +1209,14 @@ def main():
     # the tensor-core kernel with the merge fused is the whole step for up to 511 sequences; beyond that a
     # plan kernel runs ahead of it; the scalar kernel, or an unfused merge, adds the combine kernel
     fused = args.kernel == 0 and args.fuse_combine != 0
-    launches_per_step = (1 if spec.batch <= 511 else 2) if fused else 3
+    launches_per_step = ((1 if spec.batch <= 511 else 2) if fused else 3) + (1 if ctx else 0)
     traffic = None
     if args.kernel == 0 and spec.page_size == 64 and MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN:
         traffic = MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN * w.kv_tokens     # scaled from the quarter-size capture
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(3, args.warmup),
         "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "strong" if (args.shard == "kv-heads" and world > 1) else "weak", "vs_baseline": None,
+        "scaling": "strong" if (args.shard in ("kv-heads", "context") and world > 1) else "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic", "warmup_requested": args.warmup,
         "config": {"workload": args.workload, "rank0_shard": spec.name, "seed": spec.seed, "batch": spec.batch, "kv_tokens": w.kv_tokens, "page_size": spec.page_size,
                    "heads": f"{spec.num_q_heads}q/{spec.num_kv_heads}kv", "head_dim": 128, "algorithmic_bytes": nbytes,
@@ -1197,7 +1225,8 @@ def main():
                    "kv_layout": "token-major" if args.kv_layout == 1 else "head-major",
                    "parallelism": "1 gpu" if world == 1 else
                                   (f"kv-heads x{world} ({spec.num_kv_heads} KV heads per rank)" if args.shard == "kv-heads"
-                                   else f"replicas x{world}")},
+                                   else (f"context x{world} (token ranges; all-gather of (out, lse) + concur_lse_merge in the step)"
+                                         if ctx else f"replicas x{world}"))},
         "kv_tokens_per_s": (w.kv_tokens if args.shard == "kv-heads" else job_tokens) / (ms_per_step * 1e-3),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "frac_of_measured_copy": value / world / peak,

@@ -423,6 +423,26 @@ int concur_decode_attn_static(const void* q, const void* k_pages, const void* v_
                               int32_t batch, int32_t num_pages, int32_t block_table_stride,
                               int32_t page_size, void* cuda_stream);
 
+/*
+ * Merges finished attention results by their log-sum-exp: `parts` results of the SAME query rows, each
+ * over a different part of the keys, into the result over all of them --
+ *     L = ln sum_s exp(lse_s),  out = sum_s exp(lse_s - L) out_s;  a part with lse = -inf (no keys) weighs 0;
+ *     every part empty: out = 0, lse = -inf.
+ * It is the merge of the split-KV method (exact up to rounding: a re-association of the softmax sums) applied
+ * ACROSS calls: when the cache of very long sequences is spread over several GPUs by token range (context
+ * sharding), each GPU runs concur_decode_attn on its range, the (out, lse) pairs are gathered -- 260 bytes per
+ * query row and GPU -- and every GPU calls this.  The paper has no counterpart.
+ *
+ *   outs   device, bf16 [parts][rows][D], 16-byte aligned      rows = batch x Hq, D = 128
+ *   lses   device, fp32 [parts][rows], natural log, as concur_decode_attn returns it
+ *   out    device, bf16 [rows][D], 16-byte aligned;   lse  device, fp32 [rows]
+ * No handle, no workspace, no allocation; asynchronous on `cuda_stream` of the current device.  Because the
+ * parts arrive rounded to bf16, the merged result carries their rounding (2^-9 relative each) as well as its own.
+ * Errors: CONCUR_ERR_INVALID_ARG (parts < 1, rows < 0, null or misaligned pointer), CONCUR_ERR_CUDA.
+ */
+int concur_lse_merge(const void* outs, const float* lses, int32_t parts, int64_t rows,
+                     void* out, float* lse, void* cuda_stream);
+
 /* Frees the handle and any memory the library allocated for it.  NULL is accepted. */
 int concur_attn_destroy(concur_attn_t* handle);
 

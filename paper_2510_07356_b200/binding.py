@@ -51,7 +51,7 @@ EXPORTS = (
     "concur_attn_last_plan", "concur_attn_destroy", "concur_attn_strerror",
     "concur_decode_attn_static", "concur_kv_append", "concur_decode_attn_cascade", "concur_prefill_attn",
     "concur_curate", "concur_attn_plan", "concur_decode_attn_planned",
-    "concur_kv_append_layer", "concur_decode_attn_append",
+    "concur_kv_append_layer", "concur_decode_attn_append", "concur_lse_merge",
 )
 CONCUR_STATIC_MAX_BATCH = 1024
 CONCUR_STATIC_MAX_RANGES = 512
@@ -117,6 +117,8 @@ def _load() -> ctypes.CDLL:
     lib.concur_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.concur_decode_attn_append.restype = ctypes.c_int
     lib.concur_decode_attn_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i32, i32, i32, vp]
+    lib.concur_lse_merge.restype = ctypes.c_int
+    lib.concur_lse_merge.argtypes = [vp, vp, i32, ctypes.c_int64, vp, vp, vp]
     lib.concur_kv_append_layer.restype = ctypes.c_int
     lib.concur_kv_append_layer.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.concur_attn_status.restype = ctypes.c_int
@@ -298,6 +300,15 @@ def concur_decode_attn_append(handle, q, k_new, v_new, k_pages, v_pages, block_t
                                        _addr(lse), batch, num_pages, block_table_stride, stream or None)
     if check and rc != CONCUR_OK:
         raise ConcurError(rc, "concur_decode_attn_append")
+    return rc
+
+
+def concur_lse_merge(outs, lses, parts, rows, out, lse, stream=0, check=True) -> int:
+    """Merges `parts` attention results of the same query rows over different key ranges (device tensors:
+    outs bf16 [parts][rows][D], lses fp32 [parts][rows]) into out [rows][D], lse [rows]."""
+    rc = lib.concur_lse_merge(_addr(outs), _addr(lses), int(parts), int(rows), _addr(out), _addr(lse), stream or None)
+    if check and rc != CONCUR_OK:
+        raise ConcurError(rc, "concur_lse_merge")
     return rc
 
 

@@ -240,6 +240,32 @@ def shard_kv_heads(w: Workload, rank: int, world: int) -> Workload:
                     lens_host=w.lens_host, table_host=w.table_host)
 
 
+def shard_context(w: Workload, rank: int, world: int) -> Workload:
+    """Rank `rank`'s share of a workload when every sequence's tokens are spread over `world` ranks by
+    range: sequence b's pages are cut into `world` runs of (nearly) equal page counts, the rank keeps run
+    `rank` -- its table row holds those page ids, its length the tokens in them.  Pools and queries are the
+    whole workload's (a real deployment holds only its own pages; the ids stay valid here).  Slicing only."""
+    s = w.spec
+    P = s.page_size
+    assert 0 <= rank < world
+    pages = (w.lens_host.astype(np.int64) + P - 1) // P
+    lo = pages * rank // world
+    hi = pages * (rank + 1) // world
+    width = max(1, int((hi - lo).max()))
+    table = np.full((s.batch, width), -1, dtype=np.int32)
+    lens = np.zeros(s.batch, dtype=np.int32)
+    for b in range(s.batch):
+        n = int(hi[b] - lo[b])
+        table[b, :n] = w.table_host[b, lo[b]:hi[b]]
+        lens[b] = max(0, min(int(w.lens_host[b]), int(hi[b]) * P) - int(lo[b]) * P)
+    from dataclasses import replace
+    spec = replace(s, name=f"{s.name}_ctxshard{rank}of{world}", lengths=("list", [int(x) for x in lens]))
+    dev = w.q.device
+    return Workload(spec=spec, q=w.q, k_pages=w.k_pages, v_pages=w.v_pages,
+                    block_table=torch.from_numpy(table).to(dev), seq_lens=torch.from_numpy(lens).to(dev),
+                    scale=w.scale, lens_host=lens, table_host=table)
+
+
 def tiny_spec(name, lens, page_size, seed, permute=True, **kw) -> Spec:
     """A small hand-sized workload with the given context lengths."""
     return Spec(name, len(lens), page_size, ("list", list(lens)), permute_pages=permute, seed=seed, **kw)

@@ -30,6 +30,22 @@ def main():
     spec = synth.tiny_spec("ranks", (300, 1, 0, 64, 777, 1300), 16, 9100)
     w = bench.rank_workload(spec, rank, world, a.shard, "cpu")
     out, lse = oracle.decode_attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
+    if a.shard == "context":
+        # the path's one exchange step: every rank's (out, lse) over its token range is gathered on all ranks
+        # and merged by log-sum-exp (here by the oracle's merge; on a GPU by concur_lse_merge)
+        import torch
+        parts_o = [torch.empty(out.shape, dtype=torch.float64) for _ in range(world)]
+        parts_l = [torch.empty(lse.shape, dtype=torch.float64) for _ in range(world)]
+        if world > 1:
+            dist.all_gather(parts_o, torch.from_numpy(out))
+            dist.all_gather(parts_l, torch.from_numpy(lse))
+        else:
+            parts_o, parts_l = [torch.from_numpy(out)], [torch.from_numpy(lse)]
+        po = np.stack([t.numpy() for t in parts_o]); pl = np.stack([t.numpy() for t in parts_l])
+        out = np.empty_like(out); lse = np.empty_like(lse)
+        for b in range(out.shape[0]):
+            for h in range(out.shape[1]):
+                out[b, h], lse[b, h] = oracle.lse_merge(po[:, b, h], pl[:, b, h])
     ms = 1.0 + rank                              # the last rank is the slow one
     mx = bench.over_ranks([ms], "max", dev)
     sm = bench.over_ranks([float(w.algorithmic_bytes()), float(w.kv_tokens)], "sum", dev)

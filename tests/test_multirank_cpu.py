@@ -40,6 +40,45 @@ def test_kv_head_shards_of_two_ranks_put_together_equal_the_unsharded_oracle(tmp
     assert r[0]["sum_bytes"] > full.algorithmic_bytes() - 1 and r[0]["sum_bytes"] < full.algorithmic_bytes() + 4096
 
 
+def test_context_shards_of_two_ranks_gathered_and_merged_equal_the_unsharded_oracle(tmp_path):
+    import bench
+    import oracle
+    import synth
+    world = 2
+    rc = bench.spawn_ranks(WORKER, ["--gpus", str(world), "--shard", "context", "--out", str(tmp_path)], world,
+                           timeout_s=300)
+    assert rc == 0
+    r = _load(tmp_path, world)
+    full = synth.make_workload(synth.tiny_spec("ranks", (300, 1, 0, 64, 777, 1300), 16, 9100), "cpu")
+    ref_out, ref_lse = oracle.decode_attn(full.q, full.k_pages, full.v_pages, full.block_table, full.seq_lens,
+                                          full.scale)
+    for x in r:                                   # every rank ends up with the whole result
+        assert int(x["hq"]) == 64 and int(x["hkv"]) == 8
+        assert np.allclose(x["out"], ref_out, rtol=0, atol=1e-12, equal_nan=True)
+        assert np.array_equal(np.isneginf(x["lse"]), np.isneginf(ref_lse))
+        fin = np.isfinite(ref_lse)
+        assert np.allclose(x["lse"][fin], ref_lse[fin], rtol=0, atol=1e-12)
+    # the ranks' token ranges are disjoint and together the whole cache
+    assert r[0]["sum_tokens"] == float(300 + 1 + 64 + 777 + 1300)
+
+
+def test_context_shards_partition_every_sequence():
+    import synth
+    full = synth.make_workload(synth.tiny_spec("ctxp", (300, 1, 0, 64, 777, 1300, 16, 17), 16, 9101), "cpu")
+    for world in (1, 2, 3, 8):
+        shards = [synth.shard_context(full, r, world) for r in range(world)]
+        assert sum(int(s.lens_host.sum()) for s in shards) == int(full.lens_host.sum())
+        for b in range(full.spec.batch):
+            pages = []
+            for s in shards:
+                n = -(-int(s.lens_host[b]) // 16)
+                pages += s.table_host[b, :n].tolist()
+            assert pages == full.table_host[b, :-(-int(full.lens_host[b]) // 16)].tolist()
+            # only a sequence's last non-empty shard may end inside a page
+            ragged = [int(s.lens_host[b]) % 16 != 0 for s in shards if s.lens_host[b] > 0]
+            assert not any(ragged[:-1])
+
+
 def test_replica_ranks_draw_their_own_batches(tmp_path):
     import bench
     world = 2
