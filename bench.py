@@ -54,11 +54,12 @@ FALLBACK_HBM_GBS = 6650.0
 # an ncu capture of a quarter of the 64 x 16,384 configuration (page size 64, fused combine, one range per
 # CTA).  Set to None whenever that kernel changes until the counters are taken again.
 MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074892e9 + 4.929280e6) / 262144
-# The same two counters of one attn_tc_kernel launch on exactly these workloads; None for any other
+# The same two counters of one attn_tc_kernel / prefill_pair_kernel launch on exactly these workloads; None for any other
 # workload, and to be removed whenever that kernel changes until the counters are taken again.
 ATTN_TC_TRAFFIC_BYTES = {
     ("casc_16x10_pre16384_p64", "tcgen05"): 1.078966e9 + 10.120704e6,
-    ("prefill_16x2048_p64", "tcgen05"): 671.184640e6 + 506.286592e6,
+    ("prefill_16x2048_p64", "single"): 671.184640e6 + 506.286592e6,
+    ("prefill_16x2048_p64", "pair"): 671.277056e6 + 500.381440e6,
 }
 
 
@@ -89,6 +90,8 @@ def parse_args():
                     help="16/32-token pages: 1 per-lane copies (library default), 0 TMA boxes")
     ap.add_argument("--kv-layout", type=int, default=0, help="decode workloads: 0 head-major pools, 1 token-major")
     ap.add_argument("--prefix-kernel", type=int, default=0, help="cascade workloads: 0 tcgen05 prefix pass, 1 mma.sync")
+    ap.add_argument("--prefill-kernel", type=int, default=0,
+                    help="prefill workloads: 0 two query tiles per CTA over 128-token steps, 1 one tile over 64-token tiles")
     return ap.parse_args()
 
 
@@ -729,6 +732,8 @@ def run_prefill(args):
     pw = synth.make_named_prefill(args.workload, dev)
     w, spec = pw.w, pw.w.spec
     attn = P.DecodeAttention(spec.page_size, spec.batch, w.block_table.shape[1], local)
+    attn.set_option(P.CONCUR_OPT_PREFILL_KERNEL, args.prefill_kernel)
+    pf_kernel = "pair" if args.prefill_kernel == 0 else "single"
     tq = pw.total_q
     out = torch.empty((tq, spec.num_q_heads, spec.head_dim), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((tq, spec.num_q_heads), dtype=torch.float32, device=dev)
@@ -795,8 +800,8 @@ def run_prefill(args):
         "query_tokens_per_s": job_q / (ms_per_step * 1e-3),
         "roofline": {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s",
                      "frac": value / world / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": ATTN_TC_TRAFFIC_BYTES.get((spec.name, "tcgen05")),
-                     "kernel": "plan + attn_tc_kernel<prefill>", "ms": ms_per_step, "ms_min": min(step_ms)},
+                     "traffic": ATTN_TC_TRAFFIC_BYTES.get((spec.name, pf_kernel)),
+                     "kernel": "plan + " + ("prefill_pair_kernel" if pf_kernel == "pair" else "attn_tc_kernel<prefill>"), "ms": ms_per_step, "ms_min": min(step_ms)},
         "e2e": None, "gpu_launches": 2 * K, "clocks": clocks, "device_flags": flags,
     }
     print(json.dumps(line), flush=True)

@@ -123,6 +123,10 @@ typedef enum {
                                        seq_lens of a call are not written by the call right ahead of it (true
                                        of the layers of a model, whose calls differ in q, pools and out).
                                        0 (default) = calls run strictly one after the other              */
+#define CONCUR_OPT_PREFILL_KERNEL 14 /* concur_prefill_attn: 0 (default) = blocks of 32 query tokens, two tiles
+                                       of 128 accumulator rows per CTA over 128-token steps of K and V;
+                                       1 = blocks of 16 query tokens, one tile over 64-token tiles (the
+                                       pipeline the shared-prefix pass uses)                             */
 
 /* Layouts of the K and V pools (concur_attn_config_t.kv_layout). */
 #define CONCUR_KV_HEAD_MAJOR  0   /* [num_pages][Hkv][P][D]: one (page, head) tile is contiguous (default) */

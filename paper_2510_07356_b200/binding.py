@@ -44,6 +44,7 @@ CONCUR_OPT_PREFIX_KERNEL = 10
 CONCUR_OPT_SMALL_PAGE_COPY = 11
 CONCUR_OPT_WAIT_LIMIT_NS = 12
 CONCUR_OPT_OVERLAP_CALLS = 13
+CONCUR_OPT_PREFILL_KERNEL = 14
 
 EXPORTS = (
     "concur_attn_workspace_bytes", "concur_attn_create", "concur_decode_attn",

@@ -91,6 +91,7 @@ struct concur_attn {
     int32_t fuse_combine = 1;
     int32_t claim_ahead = 1 << 20;
     int32_t prefix_kernel = 0;
+    int32_t prefill_kernel = 0;
     int32_t small_page_copy = 1;
     int64_t wait_limit_ns = 2000000000ll;
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;
@@ -442,10 +443,11 @@ int concur_prefill_attn(concur_attn_t* h, const void* q, const void* k_pages, co
     PrefillParams f;
     f.q_start = q_start;
     f.total_q = total_q;
+    f.block = 0;                                                 // set by the launcher for the kernel it runs
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     h->planned_batch = -1;
     if (h->ev_before && cudaEventRecord(h->ev_before, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
-    if (launch_prefill_tc(p, f, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
+    if (launch_prefill_tc(p, f, h->prefill_kernel == 0, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     if (h->ev_after && cudaEventRecord(h->ev_after, stream) != cudaSuccess) return CONCUR_ERR_CUDA;
     return CONCUR_OK;
 }
@@ -550,6 +552,9 @@ int concur_attn_set_option(concur_attn_t* h, int32_t key, int64_t value) {
         case CONCUR_OPT_PREFIX_KERNEL:
             if (value > 1) return CONCUR_ERR_INVALID_ARG;
             h->prefix_kernel = (int32_t)value; return CONCUR_OK;
+        case CONCUR_OPT_PREFILL_KERNEL:
+            if (value > 1) return CONCUR_ERR_INVALID_ARG;
+            h->prefill_kernel = (int32_t)value; return CONCUR_OK;
         case CONCUR_OPT_SMALL_PAGE_COPY:
             if (value > 1) return CONCUR_ERR_INVALID_ARG;
             h->small_page_copy = (int32_t)value; return CONCUR_OK;

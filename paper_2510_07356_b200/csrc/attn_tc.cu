@@ -756,7 +756,7 @@ cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cuda
     return launch_attn_tc<false>(p, c, PrefillParams{}, (uint64_t)p.batch * p.hq, c.grid_ctas, stream);
 }
 
-// ---- prefill plan: blocks of 16 query tokens per sequence and their prefix sums; one unit per
+// ---- prefill plan: blocks of f.block query tokens per sequence and their prefix sums; one unit per
 //      (sequence, block, KV head)
 __global__ void __launch_bounds__(kPrefillPlanThreads) plan_prefill_kernel(DecodeParams p, PrefillParams f) {
     __shared__ int32_t warp_sums[kPrefillPlanThreads / 32];
@@ -777,7 +777,7 @@ __global__ void __launch_bounds__(kPrefillPlanThreads) plan_prefill_kernel(Decod
             int64_t q_len = (int64_t)f.q_start[b + 1] - f.q_start[b];
             if (q_len < 0) { q_len = 0; flags |= kFlagBadLen; }
             if (q_len > len) { q_len = len; flags |= kFlagBadLen; }      // more query tokens than cached tokens
-            blocks = (int32_t)((q_len + TCfg<true>::kShare - 1) / TCfg<true>::kShare);
+            blocks = (int32_t)((q_len + f.block - 1) / f.block);
         }
         int32_t v = blocks;
         #pragma unroll
@@ -811,10 +811,14 @@ __global__ void __launch_bounds__(kPrefillPlanThreads) plan_prefill_kernel(Decod
     }
 }
 
-cudaError_t launch_prefill_tc(const DecodeParams& p, const PrefillParams& f, cudaStream_t stream) {
+// pair != 0: the kernel with two query tiles per CTA (32-token blocks); else one tile (16-token blocks)
+cudaError_t launch_prefill_tc(const DecodeParams& p, const PrefillParams& f_in, int pair, cudaStream_t stream) {
+    PrefillParams f = f_in;
+    f.block = pair ? prefill_pair_block() : TCfg<true>::kShare;
     plan_prefill_kernel<<<1, kPrefillPlanThreads, 0, stream>>>(p, f);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (pair) return launch_prefill_pair(p, f, stream);
     return launch_attn_tc<true>(p, CascadeParams{}, f, (uint64_t)f.total_q * p.hq, p.grid_ctas, stream);
 }
 

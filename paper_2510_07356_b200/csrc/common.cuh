@@ -116,6 +116,7 @@ struct CascadeParams {
 struct PrefillParams {
     const int32_t* q_start;       // [batch + 1] first query token of each sequence in q / out; last entry = total_q
     int32_t total_q;
+    int32_t block;                // query tokens per unit of the kernel that runs: 16 (one tile of rows) or 32 (two)
 };
 
 // The checked build (-DCONCUR_BOUNDS) in place of a memory checker: every index a kernel computes for the
@@ -247,7 +248,9 @@ cudaError_t launch_combine(const DecodeParams& p, cudaStream_t stream);
 cudaError_t launch_plan_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 cudaError_t launch_prefix_mma(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 cudaError_t launch_prefix_tc(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
-cudaError_t launch_prefill_tc(const DecodeParams& p, const PrefillParams& f, cudaStream_t stream);
+cudaError_t launch_prefill_tc(const DecodeParams& p, const PrefillParams& f, int pair, cudaStream_t stream);
+cudaError_t launch_prefill_pair(const DecodeParams& p, const PrefillParams& f, cudaStream_t stream);
+int prefill_pair_block();
 cudaError_t launch_combine_cascade(const DecodeParams& p, const CascadeParams& c, cudaStream_t stream);
 int partial_scalar_ctas_per_sm();
 cudaError_t launch_append(const void* k_new, const void* v_new, void* k_pages, void* v_pages,

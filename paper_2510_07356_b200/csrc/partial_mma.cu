@@ -56,7 +56,8 @@ constexpr int kSmemBatch = 511;                           // sequences whose pla
 struct StageMeta {
     int32_t b, g, slot;
     int32_t n_valid;       // valid tokens in the tile (1..64); 0 = no more work
-    int32_t first, last;   // first / last tile of its segment
+    int32_t first;         // first tile of its segment
+    int32_t last;          // bit 0: last tile of its segment; bit 1: parity of the tile's flat index
     int32_t unit_start;    // flat tile index of the unit's first tile
     int32_t tiles_b;       // tiles of the whole unit
     int32_t page[4];       // small pages: pool pages of the tile's boxes (for the copy helpers)
@@ -407,7 +408,8 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
                         if (ok) {
                             StageMeta& m = meta[s];
                             m.b = sg.b; m.g = sg.g; m.slot = sg.slot; m.n_valid = n_valid;
-                            m.first = (t == sg.tile0); m.last = (t == sg.tile1 - 1);
+                            m.first = (t == sg.tile0);
+                            m.last = (t == sg.tile1 - 1 ? 1 : 0) | (((unit_start + t) & 1) << 1);
                             m.unit_start = unit_start; m.tiles_b = sg.tiles_b;
                             m.page[0] = page0; m.page[1] = page1; m.page[2] = page2; m.page[3] = page3;
                             // fused append: the sequence's last token sits in the unit's last tile
@@ -582,7 +584,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
     // Two sets: a warp's work on a tile is one dependent chain (fragment loads, 8 MMAs, shuffles, exponentials,
     // transposes, 8 MMAs) with nothing of its own to overlap it with; two sets, each with its own running
     // state, halve the time the consumer side needs per tile.
-    const int set = warp / kSetWarps;                             // this warp's set: tiles with (it & 1) == set
+    const int set = warp / kSetWarps;                             // this warp's set: tiles whose flat index has this parity
     const int tok0 = (warp % kSetWarps) * 16;                     // this warp's first token in the tile
     const uint32_t box_off = (uint32_t)(tok0 >> p.box_shift) * (uint32_t)P * kRowBytes;
     const uint32_t half_stride = (uint32_t)P * 128u;
@@ -633,7 +635,11 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
         // Both sets walk every tile's record: the segment's first tile carries its query rows (the set
         // that does not own that tile needs them for the next one) and starts both sets' states afresh,
         // and its last tile is where both meet for the merge.
-        const bool mine = (int)(it & 1u) == set;
+        // Which set takes a tile follows from the tile's place in the flat tile space, not from how many tiles
+        // this CTA happens to have seen: the grouping of a segment's sums, and with it every bit of the
+        // result, is then the same from launch to launch whichever CTA claims which range.  (Consecutive
+        // tiles still alternate; only at a jump to another range may one set get two tiles in a row.)
+        const bool mine = ((mt.last >> 1) & 1) == set;
         if (mt.first) {
             const uint32_t* qs = reinterpret_cast<const uint32_t*>(smem + s * kStageBytes + 2 * kTileBytes);
             #pragma unroll
@@ -757,7 +763,7 @@ __device__ __forceinline__ void partial_mma_body(const DecodeParams& p, const CU
         __syncwarp();
         if (lane == 0) mbar_arrive(empty(s));
 
-        if (mt.last) {
+        if (mt.last & 1) {
             // ---- merge the eight warps' states (both sets) and write the segment's result
             see_plan();
             #pragma unroll

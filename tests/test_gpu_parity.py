@@ -330,6 +330,30 @@ def test_repeated_calls_on_one_handle_are_identical(P):
     attn.close()
 
 
+@pytest.mark.parametrize("page_size,ranges,grid", [(32, 300, 0), (64, 700, 0), (16, 500, 37), (64, 0, 0)])
+def test_results_are_the_same_bits_from_launch_to_launch(P, page_size, ranges, grid):
+    # More ranges than CTAs: which CTA claims which range changes from launch to launch.  How a segment's
+    # tiles are grouped into sums must not change with it, so every launch gives the same bits.
+    lens = (4099, 0, 517, 9000, 64, 2049, 1, 12000, 333, 6000)
+    w = synth.make_workload(synth.tiny_spec("bits", lens, page_size, 4300 + page_size), "cuda:0")
+    attn = P.DecodeAttention(page_size, len(lens), w.block_table.shape[1], 0)
+    attn.set_option(P.CONCUR_OPT_NUM_RANGES, ranges)
+    attn.set_option(P.CONCUR_OPT_GRID_CTAS, grid)
+    first = None
+    for _ in range(12):
+        out, lse = attn(w.q, w.k_pages, w.v_pages, w.block_table, w.seq_lens, w.scale)
+        torch.cuda.synchronize()
+        if first is None:
+            first = (out.clone(), lse.clone())
+        else:
+            assert torch.equal(first[0].view(torch.int16), out.view(torch.int16))
+            assert torch.equal(first[1], lse)
+    assert attn.status() == 0
+    ref_out, ref_lse = oracle_sequences(to_host(w))
+    assert_parity(first[0], first[1], ref_out, ref_lse, f"p{page_size} R{ranges} grid {grid}")
+    attn.close()
+
+
 def test_a_wait_that_runs_out_returns_with_the_flag_and_leaves_the_handle_usable(P):
     # One CTA streams a whole 16,384-token sequence in two ranges that cut no unit, so its combiner
     # warp has nothing to merge and waits for a job from the kernel's start to its end, hundreds of

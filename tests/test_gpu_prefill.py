@@ -20,9 +20,22 @@ def P():
     return pkg
 
 
+# both kernels behind the entry point: 0 = two query tiles per CTA over 128-token steps (the default),
+# 1 = one tile over 64-token tiles
+KERNEL = {"value": 0}
+
+
+@pytest.fixture(autouse=True, params=[0, 1], ids=["pair", "single"])
+def prefill_kernel(request):
+    KERNEL["value"] = request.param
+    yield request.param
+    KERNEL["value"] = 0
+
+
 def run_prefill(P, pw, hq=64):
     w = pw.w
     attn = P.DecodeAttention(w.spec.page_size, w.spec.batch, w.block_table.shape[1], 0, num_q_heads=hq)
+    attn.set_option(P.CONCUR_OPT_PREFILL_KERNEL, KERNEL["value"])
     tq = pw.total_q
     out = torch.full((tq + 8, hq, 128), 7.0, dtype=torch.bfloat16, device="cuda:0")
     lse = torch.full((tq + 8, hq), 7.0, dtype=torch.float32, device="cuda:0")
@@ -97,6 +110,7 @@ def test_too_many_query_tokens_are_cut_and_flagged(P):
     w = pw.w
     short = w.seq_lens.clone(); short[1] = 20            # 50 query tokens, only 20 cached
     attn = P.DecodeAttention(64, 2, w.block_table.shape[1], 0)
+    attn.set_option(P.CONCUR_OPT_PREFILL_KERNEL, KERNEL["value"])
     out = torch.zeros_like(w.q); lse = torch.zeros((pw.total_q, 64), dtype=torch.float32, device="cuda:0")
     P.concur_prefill_attn(attn.handle, w.q, w.k_pages, w.v_pages, w.block_table, short, pw.q_start, w.scale, out, lse,
                           2, pw.total_q, w.num_pages, w.block_table.shape[1], torch.cuda.current_stream().cuda_stream)
