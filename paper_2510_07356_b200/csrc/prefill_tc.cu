@@ -359,6 +359,7 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
         if (ok && lane == 0) {
             meta[it % kPMetaRing].n = 0;                         // no more work
             mbar_arrive(meta_full(it % kPMetaRing));
+            mbar_arrive(full_k(ks));                             // the issuing warp reads records through the K barriers
         }
         if (!ok && lane == 0) {
             wait_failed(p, abort_flag, 51);
@@ -395,13 +396,15 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
         int ks = 0, vs = 0;
         uint32_t kpar = 0, vpar = 0;
         // tile B's product of the previous step, still to be issued
-        bool pend = false, pend_first = false, pend_last = false;
+        bool pend = false, pend_first = false, pend_last = false, pend_wait_v = false;
         int pend_vs = 0;
         uint32_t pend_vpar = 0;
         int32_t pend_cols = 0, pend_nvalid = 0;
         // P.V of tile t over V stage `st`: waits for V and for the tile's probabilities
-        auto issue_pv = [&](int t, int st, uint32_t stpar, int32_t ncols, int32_t nvalid, bool first) -> bool {
-            if (!warp_wait(full_v(st), stpar, abort_flag)) { site = 56; return false; }
+        auto issue_pv = [&](int t, int st, uint32_t stpar, int32_t ncols, int32_t nvalid, bool first, bool wait_v) -> bool {
+            // (a satisfied wait still costs this warp some 200 clocks, and it is the busiest role: V is waited
+            // for once per step, by the tile that reads it first)
+            if (wait_v && !warp_wait(full_v(st), stpar, abort_flag)) { site = 56; return false; }
             const uint32_t v_addr = smem_base + SM::kVOff + st * kPStageBytes;
             const int32_t used = ncols > 64 ? kPStep : 64;       // token rows this tile's product reads
             if (nvalid < used) {
@@ -454,7 +457,7 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
         };
         auto flush_pending = [&]() -> bool {
             if (!pend) return true;
-            if (!issue_pv(1, pend_vs, pend_vpar, pend_cols, pend_nvalid, pend_first)) return false;
+            if (!issue_pv(1, pend_vs, pend_vpar, pend_cols, pend_nvalid, pend_first, pend_wait_v)) return false;
             if (lane == 0) {
                 umma_commit(empty_v(pend_vs));                   // both tiles are done with that step's V
                 if (pend_last) umma_commit(pv_done(1));
@@ -465,8 +468,10 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
         };
         // A step's record, and what each tile sees of the step
         struct Rec { int32_t n, idx, cnt, nvalid, diag, cols_a, cols_b; };
+        // (the record was written before its K barrier was armed: having waited for K makes it visible, and
+        // the end marker arrives the same way)
         auto fetch = [&](uint32_t it, Rec& r) -> bool {
-            if (!warp_wait(meta_full(it % kPMetaRing), (it / kPMetaRing) & 1u, abort_flag)) { site = 52; return false; }
+            if (!warp_wait(full_k(ks), kpar, abort_flag)) { site = 54; return false; }
             const PMeta* mt = &meta[it % kPMetaRing];
             r.n = mt->n; r.idx = mt->idx; r.cnt = mt->cnt; r.nvalid = mt->nvalid; r.diag = mt->diag;
             r.cols_a = r.n ? tile_cols(r.n, 0, r.diag, r.nvalid) : 0;
@@ -487,7 +492,6 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
                     ++ofree[0];
                 }
             }
-            if (!warp_wait(full_k(ks), kpar, abort_flag)) { ok = false; site = 54; break; }
             tc_fence_after_sync();
             if (cur.cols_a > 0) issue_qk(0, ks);
             if (!flush_pending()) { ok = false; break; }
@@ -498,13 +502,14 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
             if (cur.cols_b > 0) issue_qk(1, ks);
             if (cur.idx == cur.cnt - 1 && lane == 0) umma_commit(q_empty);   // the last read of the unit's queries
             if (cur.cols_a > 0) {
-                if (!issue_pv(0, vs, vpar, cur.cols_a, cur.nvalid, cur.idx == 0)) { ok = false; break; }
+                if (!issue_pv(0, vs, vpar, cur.cols_a, cur.nvalid, cur.idx == 0, true)) { ok = false; break; }
                 if (lane == 0 && tile_last(cur.n, 0, cur.diag, cur.idx, cur.cnt)) umma_commit(pv_done(0));
                 __syncwarp();
             }
             if (cur.cols_b > 0) {
                 pend = true; pend_first = cur.idx == 0; pend_last = tile_last(cur.n, 1, cur.diag, cur.idx, cur.cnt);
                 pend_vs = vs; pend_vpar = vpar; pend_cols = cur.cols_b; pend_nvalid = cur.nvalid;
+                pend_wait_v = cur.cols_a == 0;
             } else {
                 if (lane == 0) umma_commit(empty_v(vs));         // tile B does not read this step's V
                 __syncwarp();
