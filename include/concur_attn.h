@@ -278,8 +278,9 @@ int concur_decode_attn_cascade(concur_attn_t* handle,
  *   q_start       device, int32 [batch + 1], non-decreasing, q_start[0] = 0, q_start[batch] = total_q
  *   other arguments as for concur_decode_attn
  *
- * Runs on the 5th-generation tensor cores: a unit is 16 query tokens x the query heads of one
- * KV head (up to 128 accumulator rows in tensor memory) streaming that KV head's tiles once.
+ * Runs on the 5th-generation tensor cores: a unit is 32 query tokens x the query heads of one
+ * KV head (two tiles of up to 128 accumulator rows in tensor memory) streaming that KV head's
+ * tokens once, 128 at a time (CONCUR_OPT_PREFILL_KERNEL 1: 16 query tokens, one tile, 64 at a time).
  * Asynchronous on `cuda_stream`.  q_len > seq_lens[b] is cut to seq_lens[b] and recorded as
  * CONCUR_FLAG_BAD_SEQ_LEN (the rows beyond are then not written).  Errors as for
  * concur_decode_attn; total_q < 0 or a null q_start is CONCUR_ERR_INVALID_ARG.
