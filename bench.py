@@ -53,7 +53,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one partial_mma_kernel launch divided by its KV tokens, from
 # an ncu capture of a quarter of the 64 x 16,384 configuration (page size 64, fused combine, one range per
 # CTA).  Set to None whenever that kernel changes until the counters are taken again.
-MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074892e9 + 4.929280e6) / 262144
+MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074894e9 + 5.013248e6) / 262144
 # The same two counters of one attn_tc_kernel / prefill_pair_kernel launch on exactly these workloads; None for any other
 # workload, and to be removed whenever that kernel changes until the counters are taken again.
 ATTN_TC_TRAFFIC_BYTES = {
