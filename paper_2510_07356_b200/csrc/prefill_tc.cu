@@ -331,6 +331,9 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
                     tma_load_box(dst, &map_k, my_row, my_plane, full_k(ks));
                     tma_load_box(dst + kPSlab, &map_k, my_row, my_plane + 1, full_k(ks));
                 }
+                // V of the previous step, before anything that waits for the issuing warp: at a unit's first step the
+                // wait below ends with the previous unit's last Q.K^T, and that unit's last products need this V
+                if (v_pending) { issue_v(); if (!ok) break; }
                 if (s == 0) {
                     // the unit's query rows: token j's 8 rows go to rows 8 (j % 16) .. + 7 of both halves of tile j / 16
                     ok = warp_wait(q_empty, (segs & 1u) ^ 1u, abort_flag);
@@ -347,7 +350,6 @@ prefill_pair_kernel(DecodeParams p, PrefillParams f, const __grid_constant__ CUt
                     q_inflight = true;
                     ++segs;
                 }
-                if (v_pending) { issue_v(); if (!ok) break; }
                 v_row = my_row; v_plane = my_plane; v_nbox = nbox; v_pending = true;
                 ++it;
                 if (++ks == kPKStages) { ks = 0; kpar ^= 1u; }
