@@ -59,7 +59,7 @@ MMA_P64_TRAFFIC_BYTES_PER_KV_TOKEN = (1.074894e9 + 5.013248e6) / 262144
 ATTN_TC_TRAFFIC_BYTES = {
     ("casc_16x10_pre16384_p64", "tcgen05"): 1.078966e9 + 10.120704e6,
     ("prefill_16x2048_p64", "single"): 671.184640e6 + 506.286592e6,
-    ("prefill_16x2048_p64", "pair"): 671.277056e6 + 500.381440e6,
+    ("prefill_16x2048_p64", "pair"): 671.258368e6 + 501.190400e6,
 }
 
 
