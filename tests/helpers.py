@@ -48,14 +48,15 @@ def oracle_sequences(w, seqs=None, threads=None):
     return np.concatenate([r[0] for r in res]), np.concatenate([r[1] for r in res])
 
 
-def assert_parity(out_gpu, lse_gpu, ref_out, ref_lse, what=""):
-    """out_gpu bf16 / lse_gpu fp32 torch tensors (any device) against fp64 numpy references."""
+def assert_parity(out_gpu, lse_gpu, ref_out, ref_lse, what="", out_atol=None, rel_rms_max=None):
+    """out_gpu bf16 / lse_gpu fp32 torch tensors (any device) against fp64 numpy references.
+    out_atol / rel_rms_max replace the defaults where a test derives its own (peaked rows)."""
     og = out_gpu.detach().cpu().to(torch.float64).numpy()
     lg = lse_gpu.detach().cpu().to(torch.float64).numpy()
     assert og.shape == ref_out.shape and lg.shape == ref_lse.shape, what
     assert np.isfinite(og).all(), f"{what}: non-finite output"
     err = np.abs(og - ref_out)
-    bound = OUT_ATOL + OUT_RTOL * np.abs(ref_out)
+    bound = (OUT_ATOL if out_atol is None else out_atol) + OUT_RTOL * np.abs(ref_out)
     worst = np.unravel_index(np.argmax(err - bound), err.shape)
     assert (err <= bound).all(), f"{what}: out[{worst}] = {og[worst]} vs {ref_out[worst]}"
     empty = np.isneginf(ref_lse)
@@ -64,6 +65,6 @@ def assert_parity(out_gpu, lse_gpu, ref_out, ref_lse, what=""):
     assert lerr.size == 0 or lerr.max() <= LSE_ATOL, f"{what}: lse error {lerr.max()}"
     den = np.sqrt(np.mean(ref_out ** 2))
     rel_rms = float(np.sqrt(np.mean(err ** 2)) / den) if den > 0 else 0.0
-    assert rel_rms <= REL_RMS_MAX, f"{what}: relative RMS error {rel_rms}"
+    assert rel_rms <= (REL_RMS_MAX if rel_rms_max is None else rel_rms_max), f"{what}: relative RMS error {rel_rms}"
     return {"max_abs": float(err.max()) if err.size else 0.0, "rel_rms": rel_rms,
             "lse_max_abs": float(lerr.max()) if lerr.size else 0.0}
